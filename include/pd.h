@@ -1,0 +1,152 @@
+/*
+ * pd.h -- C ABI of the per-axis 1-bit weight-delta library for NVIDIA B200 (sm_100a).
+ *
+ * A fine-tuned linear layer W_f is represented as a shared fp16 base W_b plus a
+ * bit-packed sign mask B = sign(W_f - W_b) and an fp16 scale vector v that lives on one
+ * axis: one entry per output feature ("row" axis, d_out entries) or one per input
+ * feature ("col" axis, d_in entries).  The reconstructed weight is
+ *
+ *        W_hat = W_b + v (.) B                      (paper, Method section, Eq. 1)
+ *
+ * Conventions shared by every call
+ *   - All matrices are row-major.  Weights are [d_out, d_in] (the nn.Linear layout), so the
+ *     input axis is the contiguous one.
+ *   - mask is uint32 [d_out, d_in/32]: bit k of word w of row o belongs to column 32*w + k;
+ *     bit 1 means B = +1 (dW >= 0), bit 0 means B = -1.  d_in must be a multiple of 32.
+ *   - fp16 is IEEE binary16, passed as void*.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
+ *     The library never allocates or frees device memory and keeps no pointer after a call
+ *     returns.  Scratch space comes from the caller through (workspace, workspace_bytes);
+ *     pd_workspace_bytes() tells how much a call needs.  The workspace must be 256-byte aligned.
+ *   - cuda_stream is a cudaStream_t passed as void* (NULL = the legacy default stream).  Every
+ *     call only enqueues work on that stream and returns without synchronising.
+ *   - Errors that can be seen on the host (NULL pointers, bad sizes, misalignment, a short
+ *     workspace) are returned before anything is launched.  Errors only the device can see
+ *     (a variant id out of range, a bounded wait that ran out) are latched in a device status
+ *     word inside the workspace and read back by pd_device_status().
+ *   - Input matrices, masks and scale vectors must be 16-byte aligned and ldx a multiple of 8
+ *     elements; the output y only needs its natural 2-byte alignment and any ldy >= d_out.
+ */
+#ifndef PD_H_
+#define PD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PD_OK = 0,
+    PD_ERR_INVALID_ARG = 1,       /* NULL pointer, non-positive size, bad enum value */
+    PD_ERR_UNSUPPORTED_SHAPE = 2, /* d_in not a multiple of 32, size beyond a stated maximum */
+    PD_ERR_ALIGNMENT = 3,         /* input pointer not 16-byte aligned or ldx not a multiple of 8 */
+    PD_ERR_WORKSPACE = 4,         /* workspace NULL, misaligned or smaller than pd_workspace_bytes() */
+    PD_ERR_CUDA = 5,              /* a CUDA runtime / driver call failed (launch, attribute, tensor map) */
+    PD_ERR_BAD_VARIANT = 6,       /* device saw a variant id outside [-1, V) */
+    PD_ERR_DEVICE_TIMEOUT = 7     /* a bounded device-side wait expired */
+} pd_status;
+
+typedef enum {
+    PD_AXIS_ROW = 0, /* v has d_out entries, W_hat[o,i] = W_b[o,i] + v[o] * B[o,i] */
+    PD_AXIS_COL = 1  /* v has d_in  entries, W_hat[o,i] = W_b[o,i] + v[i] * B[o,i] */
+} pd_axis;
+
+typedef enum {
+    PD_OP_PACK = 0,
+    PD_OP_LINEAR = 1,
+    PD_OP_LINEAR_MULTIVARIANT = 2,
+    PD_OP_MERGE = 3
+} pd_op;
+
+/*
+ * pd_pack_delta -- build the delta of one layer.
+ * Paper: Method section (dW = W_f - W_b, B = sign(dW)); Implementation remarks ("1 bit along
+ * input axis"); Algorithm "Per-layer compression with Row/Col selection", step 1 (pack) and
+ * steps 3 and 5 (initial scales = mean |dW| along the other axis).
+ *
+ *   w_f, w_b : in,  fp16 [d_out, d_in]
+ *   mask     : out, uint32 [d_out, d_in/32]; bit = (w_f >= w_b), i.e. sign(0) reads as +1
+ *   v_row    : out, fp16 [d_out], v_row[o] = mean_i |dW[o,i]|; may be NULL
+ *   v_col    : out, fp16 [d_in],  v_col[i] = mean_o |dW[o,i]|; may be NULL (not both NULL)
+ *
+ * The sums of |dW| are accumulated exactly (fixed point, units of 2^-24), divided once in fp64
+ * and rounded once to fp16, so the result does not depend on launch shape or summation order.
+ * Non-finite inputs are outside the contract.  Needs pd_workspace_bytes(PD_OP_PACK, ...).
+ */
+pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in,
+                        uint32_t *mask, void *v_row, void *v_col,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * pd_linear -- y = x . W_hat^T without writing W_hat to memory.
+ * Paper: Eq. 1 applied inside the forward pass (the "on-the-fly variant" of the Limitations
+ * section, which the paper names but does not build).
+ *
+ *   x    : in,  fp16 [M, d_in], row stride ldx elements
+ *   w_b  : in,  fp16 [d_out, d_in]
+ *   mask : in,  uint32 [d_out, d_in/32]; NULL means "base only" (v is ignored)
+ *   v    : in,  fp16, d_out entries (PD_AXIS_ROW) or d_in entries (PD_AXIS_COL)
+ *   y    : out, fp16 [M, d_out], row stride ldy elements
+ *
+ * fp16 products, fp32 accumulation, one rounding to fp16 at the end.  M <= 16 runs the
+ * bandwidth-bound decode kernel, larger M is cut into chunks of 16 rows up to a crossover and
+ * runs the tensor-core (tcgen05) kernel beyond it.  The tensor-core kernel needs d_out and
+ * d_in to be multiples of 8 and d_in >= 64.  Needs pd_workspace_bytes(PD_OP_LINEAR, M, ...).
+ */
+pd_status pd_linear(const void *x, int64_t M, int64_t ldx,
+                    const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
+                    int64_t d_out, int64_t d_in, void *y, int64_t ldy,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * pd_linear_multivariant -- one batch, many fine-tunes over one base.
+ * Paper: Method section ("multiple fine-tuned models ... all share the same underlying base
+ * weights"); the per-row routing is this library's reading of multi-tenant serving.
+ *
+ *   variant_ids : in, int32 [M] (device); row m uses variant ids[m]; -1 = base weights only.
+ *                 Any other value outside [0, V) latches PD_ERR_BAD_VARIANT and leaves that
+ *                 output row unspecified.
+ *   masks       : in, uint32 [V, d_out, d_in/32]
+ *   vs          : in, fp16 [V, v_stride]; variant g's scales start at vs + g*v_stride
+ *   axes        : in, HOST array of V bytes, each a pd_axis
+ *
+ * Everything else as in pd_linear.  V <= 64.
+ */
+pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids,
+                                 const void *w_b, const uint32_t *masks, const void *vs,
+                                 int64_t v_stride, const uint8_t *axes, int32_t V,
+                                 int64_t d_out, int64_t d_in, void *y, int64_t ldy,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * pd_merge -- materialise W_hat as dense fp16 weights (cold start / hot swap).
+ * Paper: Algorithm "Model-wide application from a saved delta file"; Limitations section
+ * ("add all residual terms at once ... inference identical to FP16 weights").
+ *
+ *   w_hat : out, fp16 [d_out, d_in]; w_hat[o,i] = fp16( fp32(w_b[o,i]) + (+-)fp32(v) ), the sum
+ *           rounded to fp32 and then to fp16, both to nearest even.  May alias w_b exactly.
+ * Needs no workspace.
+ */
+pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
+                   int64_t d_out, int64_t d_in, void *w_hat, void *cuda_stream);
+
+/* Bytes of workspace the given call needs (0 for PD_OP_MERGE).  M and V are ignored where they
+ * do not apply.  Returns 0 for an unknown op. */
+size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d_in);
+
+/* Synchronises the stream, reads the status word that the last pd_linear* call on this
+ * workspace latched, clears it and returns it (PD_OK when nothing was latched). */
+pd_status pd_device_status(void *workspace, void *cuda_stream);
+
+/* Human-readable name of a status code; never NULL. */
+const char *pd_status_string(pd_status status);
+
+/* Number of kernels the library has launched in this process since load (for accounting). */
+int64_t pd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PD_H_ */

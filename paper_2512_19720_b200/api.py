@@ -1,0 +1,171 @@
+"""Thin Python binding of the C ABI in include/pd.h (ctypes, argument marshalling only).
+
+Every function takes torch CUDA tensors, passes their device pointers and the current
+stream to the library and returns torch tensors.  No arithmetic of the method happens in
+Python.  If the CUDA library is missing the import fails loudly: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+AXIS_ROW = 0
+AXIS_COL = 1
+OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE = 0, 1, 2, 3
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpd.so")
+
+EXPORTS = ["pd_pack_delta", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
+           "pd_device_status", "pd_status_string", "pd_launch_count"]
+
+
+class PdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (pd_status {code})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_19720_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    p, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+    lib.pd_pack_delta.argtypes = [p, p, i64, i64, p, p, p, p, sz, p]
+    lib.pd_pack_delta.restype = ctypes.c_int
+    lib.pd_linear.argtypes = [p, i64, i64, p, p, p, ctypes.c_int, i64, i64, p, i64, p, sz, p]
+    lib.pd_linear.restype = ctypes.c_int
+    lib.pd_linear_multivariant.argtypes = [p, i64, i64, p, p, p, p, i64, p, i32, i64, i64, p, i64, p, sz, p]
+    lib.pd_linear_multivariant.restype = ctypes.c_int
+    lib.pd_merge.argtypes = [p, p, p, ctypes.c_int, i64, i64, p, p]
+    lib.pd_merge.restype = ctypes.c_int
+    lib.pd_workspace_bytes.argtypes = [ctypes.c_int, i64, i32, i64, i64]
+    lib.pd_workspace_bytes.restype = sz
+    lib.pd_device_status.argtypes = [p, p]
+    lib.pd_device_status.restype = ctypes.c_int
+    lib.pd_status_string.argtypes = [ctypes.c_int]
+    lib.pd_status_string.restype = ctypes.c_char_p
+    lib.pd_launch_count.argtypes = []
+    lib.pd_launch_count.restype = i64
+    return lib
+
+
+lib = _load()
+
+
+def status_string(code: int) -> str:
+    return lib.pd_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(lib.pd_launch_count())
+
+
+def workspace_bytes(op: int, m: int = 0, n_variants: int = 0, d_out: int = 0, d_in: int = 0) -> int:
+    return int(lib.pd_workspace_bytes(op, m, n_variants, d_out, d_in))
+
+
+_ws_cache: dict = {}
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    """A cached scratch tensor of at least nbytes on `device` (torch allocations are 512-byte aligned)."""
+    key = (device.type, device.index)
+    ws = _ws_cache.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.zeros(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _ws_cache[key] = ws
+    return ws
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise PdError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _want(t, dtype, name):
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError(f"{name} must be a CUDA tensor of {dtype}")
+
+
+def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None, v_col=None, workspace=None):
+    """mask uint32-as-int32 [d_out, d_in/32], v_row fp16 [d_out] | None, v_col fp16 [d_in] | None."""
+    _want(w_f, torch.float16, "w_f"), _want(w_b, torch.float16, "w_b")
+    assert w_f.shape == w_b.shape and w_f.is_contiguous() and w_b.is_contiguous()
+    d_out, d_in = w_b.shape
+    dev = w_b.device
+    if mask is None:
+        mask = torch.empty((d_out, d_in // 32), dtype=torch.int32, device=dev)
+    if want_row and v_row is None:
+        v_row = torch.empty(d_out, dtype=torch.float16, device=dev)
+    if want_col and v_col is None:
+        v_col = torch.empty(d_in, dtype=torch.float16, device=dev)
+    need = workspace_bytes(OP_PACK, 0, 0, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, dev)
+    _check(lib.pd_pack_delta(_ptr(w_f), _ptr(w_b), d_out, d_in, _ptr(mask), _ptr(v_row if want_row else None),
+                             _ptr(v_col if want_col else None), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "pd_pack_delta")
+    return mask, (v_row if want_row else None), (v_col if want_col else None)
+
+
+def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None):
+    """y fp16 [M, d_out] = x . (W_b + v (.) B)^T; mask None = base weights only."""
+    _want(x, torch.float16, "x"), _want(w_b, torch.float16, "w_b")
+    assert x.dim() == 2 and x.stride(1) == 1 and w_b.is_contiguous()
+    m, d_in = x.shape
+    d_out = w_b.shape[0]
+    assert w_b.shape[1] == d_in
+    if y is None:
+        y = torch.empty((m, d_out), dtype=torch.float16, device=x.device)
+    need = workspace_bytes(OP_LINEAR, m, 0, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, x.device)
+    _check(lib.pd_linear(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
+                         y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pd_linear")
+    return y
+
+
+def pd_linear_multivariant(x, variant_ids, w_b, masks, vs, axes, y=None, workspace=None):
+    """Row m of x uses variant variant_ids[m] (-1 = base only).  masks [V, d_out, d_in/32], vs fp16
+    [V, v_stride], axes: sequence of V axis codes (host)."""
+    _want(x, torch.float16, "x"), _want(w_b, torch.float16, "w_b"), _want(variant_ids, torch.int32, "variant_ids")
+    assert x.dim() == 2 and x.stride(1) == 1 and w_b.is_contiguous() and masks.is_contiguous() and vs.is_contiguous()
+    m, d_in = x.shape
+    d_out = w_b.shape[0]
+    n_var = masks.shape[0]
+    if y is None:
+        y = torch.empty((m, d_out), dtype=torch.float16, device=x.device)
+    axes_arr = (ctypes.c_uint8 * n_var)(*[int(a) for a in axes])
+    need = workspace_bytes(OP_LINEAR_MULTIVARIANT, m, n_var, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, x.device)
+    _check(lib.pd_linear_multivariant(_ptr(x), m, x.stride(0), _ptr(variant_ids), _ptr(w_b), _ptr(masks), _ptr(vs),
+                                      vs.stride(0), axes_arr, n_var, d_out, d_in, _ptr(y), y.stride(0), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _stream()), "pd_linear_multivariant")
+    return y
+
+
+def pd_merge(w_b, mask, v, axis, w_hat=None):
+    """Dense fp16 W_hat = fp16(fp32(W_b) +- fp32(v)); w_hat may be w_b itself."""
+    _want(w_b, torch.float16, "w_b")
+    assert w_b.is_contiguous()
+    d_out, d_in = w_b.shape
+    if w_hat is None:
+        w_hat = torch.empty_like(w_b)
+    _check(lib.pd_merge(_ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(w_hat), _stream()), "pd_merge")
+    return w_hat
+
+
+def pd_device_status(workspace=None, device=None) -> int:
+    """Synchronise the current stream and return the status a linear call latched (0 = ok)."""
+    ws = workspace if workspace is not None else _workspace(256, device or torch.device("cuda", torch.cuda.current_device()))
+    return int(lib.pd_device_status(_ptr(ws), _stream()))

@@ -1,0 +1,209 @@
+// C ABI of the pd library: argument checks, workspace layout, dispatch.  No device memory is
+// allocated here; everything runs on the caller's stream.
+#include <climits>
+
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+constexpr int kMaxVariants = 64;
+constexpr int kGroupThreads = 1024;
+
+// workspace layout of the linear calls:
+//   [0, 256)                status words
+//   [256, 256 + 4*(V+2))    group offsets (rounded up to 512 bytes)
+//   [768, 768 + 4*M)        row_index
+constexpr size_t kOffsetsBytes = 512;
+
+__global__ void __launch_bounds__(kGroupThreads)
+group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict__ offsets,
+                  int *__restrict__ row_index, uint32_t *__restrict__ status) {
+    __shared__ int warp_sums[kGroupThreads / 32];
+    __shared__ int s_base;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        s_base = 0;
+        offsets[0] = 0;
+    }
+    for (int i = threadIdx.x; i < M; i += kGroupThreads) {
+        const int id = ids[i];
+        if (id < -1 || id >= V) latch_error(status, PD_ERR_BAD_VARIANT, static_cast<uint32_t>(i));
+    }
+    __syncthreads();
+    for (int grp = 0; grp <= V; ++grp) {
+        const int want = (grp == V) ? -1 : grp;
+        for (int c0 = 0; c0 < M; c0 += kGroupThreads) {
+            const int i = c0 + threadIdx.x;
+            const bool hit = i < M && ids[i] == want;
+            const unsigned ballot = __ballot_sync(0xffffffffu, hit);
+            if (lane == 0) warp_sums[warp] = __popc(ballot);
+            __syncthreads();
+            int before = 0, total = 0;
+            for (int w = 0; w < kGroupThreads / 32; ++w) {
+                const int c = warp_sums[w];
+                before += (w < warp) ? c : 0;
+                total += c;
+            }
+            const int base = s_base;
+            if (hit) row_index[base + before + __popc(ballot & ((1u << lane) - 1u))] = i;
+            __syncthreads();
+            if (threadIdx.x == 0) s_base = base + total;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) offsets[grp + 1] = s_base;
+    }
+}
+
+pd_status check_matrix_args(const void *x, int64_t M, int64_t ldx, const void *w_b, int64_t d_out, int64_t d_in,
+                            const void *y, int64_t ldy) {
+    if (!x || !w_b || !y || M <= 0 || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || d_out > INT_MAX / 2 || d_in > INT_MAX / 2 || M > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (ldx < d_in || ldy < d_out) return PD_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_b) || (reinterpret_cast<uintptr_t>(y) & 1u) || ldx % 8 != 0) return PD_ERR_ALIGNMENT;
+    return PD_OK;
+}
+
+}  // namespace
+
+pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,
+                            cudaStream_t stream) {
+    group_rows_kernel<<<1, kGroupThreads, 0, stream>>>(ids, M, V, offsets, row_index, status);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace pd
+
+using namespace pd;
+
+extern "C" {
+
+size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d_in) {
+    switch (op) {
+        case PD_OP_PACK:
+            return kStatusBytes + round_up(sizeof(unsigned long long) * static_cast<size_t>(d_out + d_in), 256);
+        case PD_OP_LINEAR:
+            return kStatusBytes;
+        case PD_OP_LINEAR_MULTIVARIANT:
+            (void)V;
+            return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M > 0 ? M : 0), 256);
+        case PD_OP_MERGE:
+        default:
+            return 0;
+    }
+}
+
+const char *pd_status_string(pd_status s) {
+    switch (s) {
+        case PD_OK: return "ok";
+        case PD_ERR_INVALID_ARG: return "invalid argument";
+        case PD_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case PD_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+        case PD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case PD_ERR_CUDA: return "CUDA call failed";
+        case PD_ERR_BAD_VARIANT: return "variant id out of range";
+        case PD_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int64_t pd_launch_count(void) { return g_launches.load(); }
+
+pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in, uint32_t *mask, void *v_row,
+                        void *v_col, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!w_f || !w_b || !mask || (!v_row && !v_col) || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || d_out > INT_MAX / 2 || d_in > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(w_f) || !aligned16(w_b) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_PACK, 0, 0, d_out, d_in))
+        return PD_ERR_WORKSPACE;
+    auto *sums = reinterpret_cast<unsigned long long *>(static_cast<unsigned char *>(workspace) + kStatusBytes);
+    return launch_pack(static_cast<const __half *>(w_f), static_cast<const __half *>(w_b), d_out, d_in, mask,
+                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis, int64_t d_out, int64_t d_in,
+                   void *w_hat, void *cuda_stream) {
+    if (!w_b || !mask || !v || !w_hat || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (axis != PD_AXIS_ROW && axis != PD_AXIS_COL) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || d_out > INT_MAX / 2 || d_in > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(w_b) || !aligned16(w_hat) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
+    if (axis == PD_AXIS_COL && !aligned16(v)) return PD_ERR_ALIGNMENT;
+    return launch_merge(static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis, d_out, d_in,
+                        static_cast<__half *>(w_hat), static_cast<cudaStream_t>(cuda_stream));
+}
+
+pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                    pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                    size_t workspace_bytes, void *cuda_stream) {
+    pd_status st = check_matrix_args(x, M, ldx, w_b, d_out, d_in, y, ldy);
+    if (st != PD_OK) return st;
+    if (axis != PD_AXIS_ROW && axis != PD_AXIS_COL) return PD_ERR_INVALID_ARG;
+    if (mask && !v) return PD_ERR_INVALID_ARG;
+    if (mask && (!aligned16(mask) || !aligned16(v))) return PD_ERR_ALIGNMENT;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_LINEAR, M, 0, d_out, d_in))
+        return PD_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const __half *xh = static_cast<const __half *>(x);
+    __half *yh = static_cast<__half *>(y);
+    for (int64_t m0 = 0; m0 < M; m0 += 16) {
+        const int rows = static_cast<int>(M - m0 < 16 ? M - m0 : 16);
+        st = launch_gemv(xh + m0 * ldx, rows, ldx, static_cast<const __half *>(w_b), mask,
+                         static_cast<const __half *>(v), axis, d_out, d_in, yh + m0 * ldy, ldy, nullptr, nullptr, 0,
+                         stream);
+        if (st != PD_OK) return st;
+    }
+    return PD_OK;
+}
+
+pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
+                                 const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes,
+                                 int32_t V, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                                 size_t workspace_bytes, void *cuda_stream) {
+    pd_status st = check_matrix_args(x, M, ldx, w_b, d_out, d_in, y, ldy);
+    if (st != PD_OK) return st;
+    if (!variant_ids || !masks || !vs || !axes || V <= 0) return PD_ERR_INVALID_ARG;
+    if (V > kMaxVariants) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(masks) || !aligned16(vs) || v_stride % 8 != 0) return PD_ERR_ALIGNMENT;
+    for (int g = 0; g < V; ++g) {
+        if (axes[g] != PD_AXIS_ROW && axes[g] != PD_AXIS_COL) return PD_ERR_INVALID_ARG;
+        if (v_stride < (axes[g] == PD_AXIS_ROW ? d_out : d_in)) return PD_ERR_INVALID_ARG;
+    }
+    if (!workspace || !aligned256(workspace) ||
+        workspace_bytes < pd_workspace_bytes(PD_OP_LINEAR_MULTIVARIANT, M, V, d_out, d_in))
+        return PD_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    auto *base = static_cast<unsigned char *>(workspace);
+    auto *status = reinterpret_cast<uint32_t *>(base);
+    int *offsets = reinterpret_cast<int *>(base + kStatusBytes);
+    int *row_index = reinterpret_cast<int *>(base + kStatusBytes + kOffsetsBytes);
+    if (cudaMemsetAsync(status, 0, kStatusBytes, stream) != cudaSuccess) return PD_ERR_CUDA;
+    st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, stream);
+    if (st != PD_OK) return st;
+    const __half *xh = static_cast<const __half *>(x);
+    const __half *vh = static_cast<const __half *>(vs);
+    const int64_t mask_words = d_out * (d_in / 32);
+    for (int g = 0; g <= V; ++g) {
+        const bool base_only = (g == V);
+        st = launch_gemv(xh, 0, ldx, static_cast<const __half *>(w_b), base_only ? nullptr : masks + g * mask_words,
+                         base_only ? nullptr : vh + g * v_stride, base_only ? PD_AXIS_ROW : axes[g], d_out, d_in,
+                         static_cast<__half *>(y), ldy, row_index, offsets, g, stream);
+        if (st != PD_OK) return st;
+    }
+    return PD_OK;
+}
+
+pd_status pd_device_status(void *workspace, void *cuda_stream) {
+    if (!workspace) return PD_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t words[2] = {0, 0};
+    if (cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return PD_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return PD_ERR_CUDA;
+    if (words[0] != 0) {
+        if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return PD_ERR_CUDA;
+    }
+    return static_cast<pd_status>(words[0]);
+}
+
+}  // extern "C"

@@ -1,0 +1,49 @@
+// Shared host/device helpers of the pd library (sm_100a only).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "pd.h"
+
+namespace pd {
+
+// First bytes of every workspace: words the device latches errors into.
+//   word 0: status (0 = ok, else a pd_status value), word 1: detail (bad id, or stage that timed out)
+constexpr size_t kStatusBytes = 256;
+
+extern std::atomic<int64_t> g_launches;
+
+inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline pd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PD_OK : PD_ERR_CUDA; }
+
+__device__ __forceinline__ void latch_error(uint32_t *status, uint32_t code, uint32_t detail) {
+    if (atomicCAS(status, 0u, code) == 0u) status[1] = detail;
+}
+
+// --- launchers implemented in the .cu files (all enqueue on `stream`, none synchronises) ---
+pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
+                      __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream);
+pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
+                       int64_t d_in, __half *w_hat, cudaStream_t stream);
+
+// M <= 16 tokens (mask == nullptr: base weights only).  With group_offsets != nullptr the tokens are
+// rows row_index[group_offsets[group] .. group_offsets[group+1]) of x / y (any count, read on the device).
+pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask,
+                      const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
+                      const int *row_index, const int *group_offsets, int group, cudaStream_t stream);
+
+// Stable bucket sort of token rows by variant id: offsets[g] .. offsets[g+1] index row_index for
+// variant g (g = 0..V-1), offsets[V] .. offsets[V+1] the rows with id -1.  Other ids latch an error.
+pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,
+                            cudaStream_t stream);
+
+}  // namespace pd

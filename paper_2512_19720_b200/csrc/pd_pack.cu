@@ -1,0 +1,256 @@
+// pack: sign mask of W_f - W_b plus the exact per-axis sums of |W_f - W_b|, and
+// merge: W_hat = fp16(fp32(W_b) +- fp32(v)).  Both are single-pass streaming kernels bound by HBM
+// (4.125 bytes per weight element each).
+//
+// Tile shape for both: a CTA of 8 warps covers 64 rows x 256 columns; a warp owns one row at a
+// time, a lane owns 8 consecutive columns (one 128-bit load per matrix), so four neighbouring
+// lanes form one 32-bit mask word.
+#include "pd_common.cuh"
+
+namespace pd {
+
+std::atomic<int64_t> g_launches{0};
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kTileRows = 64;
+constexpr int kTileCols = 256;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// same without the read-only path: merge may write its output over its input
+__device__ __forceinline__ uint4 ldg_stream_coherent(const uint4 *p) {
+    uint4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
+
+__device__ __forceinline__ void stg_stream(uint4 *p, uint4 v) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ __half2 as_half2(uint32_t u) { return *reinterpret_cast<__half2 *>(&u); }
+
+// Signed value of a binary16 in units of 2^-24 (every finite binary16 is an integer number of them).
+__device__ __forceinline__ long long half_units(uint32_t h) {
+    const uint32_t e = (h >> 10) & 31u, m = h & 1023u;
+    const long long mag = e ? (static_cast<long long>(m | 1024u) << (e - 1u)) : static_cast<long long>(m);
+    return (h & 0x8000u) ? -mag : mag;
+}
+
+// |a - b| in units of 2^-24 for two binary16 values both below 0.25 in magnitude: the fp32
+// difference is exact (23 bits), and adding 0.5 places it where one fp32 ulp is 2^-24.
+__device__ __forceinline__ uint32_t abs_diff_units_small(float a, float b) {
+    return __float_as_uint(fabsf(__fsub_rn(a, b)) + 0.5f) - 0x3f000000u;
+}
+
+template <bool ROW, bool COL>
+__global__ void __launch_bounds__(kThreads)
+pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_out, int d_in, int tiles_c,
+            uint32_t *__restrict__ mask, unsigned long long *__restrict__ row_sum,
+            unsigned long long *__restrict__ col_sum) {
+    __shared__ uint32_t s_col[COL ? (kThreads / 32) * kTileCols : 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int tile_r = blockIdx.x / tiles_c, tile_c = blockIdx.x - tile_r * tiles_c;
+    const int col0 = tile_c * kTileCols + lane * 8;
+    const int row0 = tile_r * kTileRows;
+    const bool col_ok = col0 < d_in;
+    const int words = d_in >> 5;
+
+    uint32_t cacc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) cacc[j] = 0;
+
+#pragma unroll 4
+    for (int rr = warp; rr < kTileRows; rr += kThreads / 32) {
+        const int o = row0 + rr;
+        if (o >= d_out) break;  // warp-uniform
+        uint32_t bits = 0, fast_sum = 0;
+        unsigned long long slow_sum = 0;
+        bool slow = false;
+        if (col_ok) {
+            const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
+            const uint4 a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
+            const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+            uint32_t big = 0;
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                // bit = (w_f >= w_b): exact on binary16, false for NaN, true for -0 vs +0
+                const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p])) & 0x00010001u;
+                bits |= ((ge | (ge >> 15)) & 3u) << (2 * p);
+                big |= ((a[p] & 0x7fff7fffu) + 0x4c004c00u) | ((b[p] & 0x7fff7fffu) + 0x4c004c00u);
+            }
+            slow = (big & 0x80008000u) != 0;  // some |w| >= 0.25 (0x3400)
+            if (!slow) {
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                    const float2 fa = __half22float2(as_half2(a[p])), fb = __half22float2(as_half2(b[p]));
+                    const uint32_t u0 = abs_diff_units_small(fa.x, fb.x), u1 = abs_diff_units_small(fa.y, fb.y);
+                    if (COL) {
+                        cacc[2 * p] += u0;
+                        cacc[2 * p + 1] += u1;
+                    }
+                    fast_sum += u0 + u1;
+                }
+            } else {
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const long long d = half_units((a[p] >> (16 * h)) & 0xffffu) -
+                                            half_units((b[p] >> (16 * h)) & 0xffffu);
+                        const unsigned long long u = static_cast<unsigned long long>(d < 0 ? -d : d);
+                        slow_sum += u;
+                        if (COL) atomicAdd(col_sum + col0 + 2 * p + h, u);
+                    }
+                }
+            }
+        }
+        uint32_t word = bits << (8 * (lane & 3));
+        word |= __shfl_xor_sync(kFull, word, 1);
+        word |= __shfl_xor_sync(kFull, word, 2);
+        if ((lane & 3) == 0 && col_ok) mask[static_cast<size_t>(o) * words + (col0 >> 5)] = word;
+        if (ROW) {
+            // each lane adds at most 8 * 2^23 units on the fast path, so the 32-lane sum fits 32 bits
+            unsigned long long total = __reduce_add_sync(kFull, fast_sum);
+            if (__any_sync(kFull, slow)) {
+#pragma unroll
+                for (int s = 16; s > 0; s >>= 1) slow_sum += __shfl_xor_sync(kFull, slow_sum, s);
+                total += slow_sum;
+            }
+            if (lane == 0) atomicAdd(row_sum + o, total);
+        }
+    }
+    if (COL) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s_col[warp * kTileCols + lane * 8 + j] = cacc[j];
+        __syncthreads();
+        const int c = tile_c * kTileCols + threadIdx.x;
+        if (c < d_in) {
+            uint32_t t = 0;  // <= 64 rows * 2^23 units
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) t += s_col[w * kTileCols + threadIdx.x];
+            atomicAdd(col_sum + c, static_cast<unsigned long long>(t));
+        }
+    }
+}
+
+// mean = (sum * 2^-24) / n with one fp64 division, then one rounding to binary16
+__global__ void pack_finalize_kernel(const unsigned long long *__restrict__ row_sum,
+                                     const unsigned long long *__restrict__ col_sum, int d_out, int d_in,
+                                     __half *__restrict__ v_row, __half *__restrict__ v_col) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool is_row = idx < d_out;
+    const int j = is_row ? idx : idx - d_out;
+    if (!is_row && j >= d_in) return;
+    __half *dst = is_row ? v_row : v_col;
+    if (dst == nullptr) return;
+    const unsigned long long s = is_row ? row_sum[j] : col_sum[j];
+    const double q = __ddiv_rn(static_cast<double>(s), static_cast<double>(is_row ? d_in : d_out)) *
+                     5.9604644775390625e-08;  // 2^-24, exact scaling
+    unsigned short h;
+    asm("cvt.rn.f16.f64 %0, %1;" : "=h"(h) : "d"(q));
+    reinterpret_cast<unsigned short *>(dst)[j] = h;
+}
+
+template <int AXIS>
+__global__ void __launch_bounds__(kThreads)
+merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *__restrict__ v, int d_out, int d_in,
+             int tiles_c, uint4 *w_hat) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int tile_r = blockIdx.x / tiles_c, tile_c = blockIdx.x - tile_r * tiles_c;
+    const int col0 = tile_c * kTileCols + lane * 8;
+    const int row0 = tile_r * kTileRows;
+    if (col0 >= d_in) return;
+    const int words = d_in >> 5;
+    float vf[8];
+    if (AXIS == PD_AXIS_COL) {
+        const uint4 vv = *reinterpret_cast<const uint4 *>(v + col0);
+        const uint32_t u[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float2 f = __half22float2(as_half2(u[p]));
+            vf[2 * p] = f.x;
+            vf[2 * p + 1] = f.y;
+        }
+    }
+#pragma unroll 4
+    for (int rr = warp; rr < kTileRows; rr += kThreads / 32) {
+        const int o = row0 + rr;
+        if (o >= d_out) break;
+        const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
+        const uint4 w4 = ldg_stream_coherent(w_b + idx);
+        const uint32_t word = __ldg(mask + static_cast<size_t>(o) * words + (col0 >> 5));
+        const uint32_t nbits = ~(word >> (8 * (lane & 3)));  // bit set -> B = -1
+        if (AXIS == PD_AXIS_ROW) {
+            const float s = __half2float(v[o]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) vf[j] = s;
+        }
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        uint32_t r[4];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float2 f = __half22float2(as_half2(w[p]));
+            const float s0 = __uint_as_float(__float_as_uint(vf[2 * p]) ^ (((nbits >> (2 * p)) & 1u) << 31));
+            const float s1 = __uint_as_float(__float_as_uint(vf[2 * p + 1]) ^ (((nbits >> (2 * p + 1)) & 1u) << 31));
+            const __half2 h = __floats2half2_rn(__fadd_rn(f.x, s0), __fadd_rn(f.y, s1));
+            r[p] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        stg_stream(w_hat + idx, make_uint4(r[0], r[1], r[2], r[3]));
+    }
+}
+
+}  // namespace
+
+pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
+                      __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream) {
+    unsigned long long *row_sum = sums, *col_sum = sums + d_out;
+    if (cudaMemsetAsync(sums, 0, sizeof(unsigned long long) * static_cast<size_t>(d_out + d_in), stream) != cudaSuccess)
+        return PD_ERR_CUDA;
+    const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
+    const int64_t tiles = ((d_out + kTileRows - 1) / kTileRows) * tiles_c;
+    const dim3 grid(static_cast<unsigned>(tiles)), block(kThreads);
+    const uint4 *a = reinterpret_cast<const uint4 *>(w_f), *b = reinterpret_cast<const uint4 *>(w_b);
+    const int n_out = static_cast<int>(d_out), n_in = static_cast<int>(d_in);
+    if (v_row && v_col)
+        pack_kernel<true, true><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    else if (v_row)
+        pack_kernel<true, false><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    else
+        pack_kernel<false, true><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    const int n = static_cast<int>(d_out + d_in);
+    pack_finalize_kernel<<<(n + 255) / 256, 256, 0, stream>>>(row_sum, col_sum, n_out, n_in, v_row, v_col);
+    count_launch(2);
+    return cuda_ok(cudaGetLastError());
+}
+
+pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
+                       int64_t d_in, __half *w_hat, cudaStream_t stream) {
+    const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
+    const int64_t tiles = ((d_out + kTileRows - 1) / kTileRows) * tiles_c;
+    const dim3 grid(static_cast<unsigned>(tiles)), block(kThreads);
+    const uint4 *b = reinterpret_cast<const uint4 *>(w_b);
+    uint4 *out = reinterpret_cast<uint4 *>(w_hat);
+    if (axis == PD_AXIS_ROW)
+        merge_kernel<PD_AXIS_ROW><<<grid, block, 0, stream>>>(b, mask, v, (int)d_out, (int)d_in, tiles_c, out);
+    else
+        merge_kernel<PD_AXIS_COL><<<grid, block, 0, stream>>>(b, mask, v, (int)d_out, (int)d_in, tiles_c, out);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace pd

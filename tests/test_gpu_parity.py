@@ -1,0 +1,300 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Pack and merge must be bit-exact; linear outputs must satisfy
+max|y - y_ref| / max|y_ref| <= 5e-3 (fp16 products, fp32 accumulation, one fp16 rounding)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pd_oracle as orc
+from paper_2512_19720_b200 import synth
+
+pytestmark = pytest.mark.gpu
+ROW, COL = 0, 1
+TOL = 5e-3
+
+
+@pytest.fixture(scope="module")
+def api():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2512_19720_b200 import api as _api
+    return _api
+
+
+def dev(a):
+    if a.dtype == np.uint32:
+        a = a.view(np.int32)
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    a = t.detach().cpu().numpy()
+    return a.view(np.uint32) if a.dtype == np.int32 else a
+
+
+def bits(a):
+    return np.ascontiguousarray(a).view(np.uint16)
+
+
+def rel_err(y, y_ref):
+    return float(np.max(np.abs(y.astype(np.float64) - y_ref)) / np.max(np.abs(y_ref)))
+
+
+class Layer:
+    """One synthetic (W_b, W_f) pair with the oracle's pack results, on host and device."""
+
+    def __init__(self, d_out, d_in, seed=0, ft_seed=None, sigma=1e-3):
+        self.d_out, self.d_in = d_out, d_in
+        self.w_b = synth.gen_base(d_out, d_in, seed)
+        self.w_f = synth.gen_finetuned(self.w_b, 1000 + seed if ft_seed is None else ft_seed, sigma)
+        self.mask, self.v_row, self.v_col = orc.pack(self.w_f, self.w_b)
+        self.d_w_b, self.d_w_f = dev(self.w_b), dev(self.w_f)
+        self.d_mask, self.d_v_row, self.d_v_col = dev(self.mask), dev(self.v_row), dev(self.v_col)
+
+    def v(self, axis):
+        return self.v_row if axis == ROW else self.v_col
+
+    def d_v(self, axis):
+        return self.d_v_row if axis == ROW else self.d_v_col
+
+
+_layers = {}
+
+
+def layer(d_out, d_in, seed=0):
+    key = (d_out, d_in, seed)
+    if key not in _layers:
+        if len(_layers) > 3:
+            _layers.clear()
+            torch.cuda.empty_cache()
+        _layers[key] = Layer(d_out, d_in, seed)
+    return _layers[key]
+
+
+# ------------------------------------------------------------------ pack
+PACK_SHAPES = [(1024, 1024), (64, 32), (1, 32), (65, 96), (200, 1056), (130, 288), (4096, 4096), (4096, 11008)]
+
+
+@pytest.mark.parametrize("d_out,d_in", PACK_SHAPES)
+def test_pack_bit_exact(api, d_out, d_in):
+    L = layer(d_out, d_in)
+    guard = 64
+    mask = torch.full((d_out * (d_in // 32) + 2 * guard,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    v_row = torch.full((d_out + 2 * guard,), 123.0, dtype=torch.float16, device="cuda")
+    v_col = torch.full((d_in + 2 * guard,), 123.0, dtype=torch.float16, device="cuda")
+    m_view = mask[guard:-guard].view(d_out, d_in // 32)
+    api.pd_pack_delta(L.d_w_f, L.d_w_b, mask=m_view, v_row=v_row[guard:-guard], v_col=v_col[guard:-guard])
+    torch.cuda.synchronize()
+    assert np.array_equal(host(m_view), L.mask)
+    assert np.array_equal(bits(host(v_row[guard:-guard])), bits(L.v_row))
+    assert np.array_equal(bits(host(v_col[guard:-guard])), bits(L.v_col))
+    for buf, fill in ((mask, 0x5A5A5A5A), (v_row, 123.0), (v_col, 123.0)):  # canaries untouched
+        assert bool((buf[:guard] == fill).all()) and bool((buf[-guard:] == fill).all())
+    # one axis at a time gives the same answers, and a second run is bit-identical
+    m2, vr2, none = api.pd_pack_delta(L.d_w_f, L.d_w_b, want_col=False)
+    m3, none2, vc3 = api.pd_pack_delta(L.d_w_f, L.d_w_b, want_row=False)
+    torch.cuda.synchronize()
+    assert none is None and none2 is None
+    assert np.array_equal(host(m2), L.mask) and np.array_equal(host(m3), L.mask)
+    assert np.array_equal(bits(host(vr2)), bits(L.v_row)) and np.array_equal(bits(host(vc3)), bits(L.v_col))
+
+
+def test_pack_large_magnitudes_take_the_exact_wide_path(api):
+    # weights up to +-60000 and subnormals: the 64-bit fixed-point path must still be exact
+    rng = np.random.default_rng(5)
+    d_out, d_in = 96, 320
+    w_b = (rng.standard_normal((d_out, d_in)) * rng.choice([1e-6, 1e-3, 0.3, 40.0, 9000.0], size=(d_out, d_in))).astype(np.float16)
+    w_f = (w_b.astype(np.float64) + rng.standard_normal((d_out, d_in)) * rng.choice([1e-7, 1e-2, 5.0], size=(d_out, d_in))).astype(np.float16)
+    w_f[3, 7] = w_b[3, 7]
+    w_b[5, 9], w_f[5, 9] = np.float16(0.0), np.float16(-0.0)
+    mask, v_row, v_col = orc.pack(w_f, w_b)
+    m, vr, vc = api.pd_pack_delta(dev(w_f), dev(w_b))
+    torch.cuda.synchronize()
+    assert np.array_equal(host(m), mask)
+    assert np.array_equal(bits(host(vr)), bits(v_row))
+    assert np.array_equal(bits(host(vc)), bits(v_col))
+
+
+# ------------------------------------------------------------------ merge
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in", [(1024, 1024), (65, 96), (200, 1056), (4096, 4096), (11008, 4096)])
+def test_merge_bit_exact(api, d_out, d_in, axis):
+    L = layer(d_out, d_in)
+    ref = orc.merge(L.w_b, L.mask, L.v(axis), axis)
+    out = api.pd_merge(L.d_w_b, L.d_mask, L.d_v(axis), axis)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(host(out)), bits(ref))
+    # in place over the base
+    w = L.d_w_b.clone()
+    api.pd_merge(w, L.d_mask, L.d_v(axis), axis, w_hat=w)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(host(w)), bits(ref))
+
+
+def test_merge_wide_exponent_range(api):
+    rng = np.random.default_rng(6)
+    d_out, d_in = 64, 256
+    w_b = rng.integers(0, 0x7800, size=(d_out, d_in)).astype(np.uint16)
+    w_b ^= (rng.integers(0, 2, size=(d_out, d_in)).astype(np.uint16) << 15)
+    w_b = w_b.view(np.float16)
+    mask = rng.integers(0, 2 ** 32, size=(d_out, d_in // 32), dtype=np.uint64).astype(np.uint32)
+    for axis, n in ((ROW, d_out), (COL, d_in)):
+        v = rng.integers(0, 0x5000, size=n).astype(np.uint16).view(np.float16)
+        ref = orc.merge(w_b, mask, v, axis)
+        out = api.pd_merge(dev(w_b), dev(mask), dev(v), axis)
+        torch.cuda.synchronize()
+        assert np.array_equal(bits(host(out)), bits(ref))
+
+
+def test_pack_merge_round_trip_on_device(api):
+    L = layer(1024, 1024)
+    w_hat = api.pd_merge(L.d_w_b, L.d_mask, L.d_v_row, ROW)
+    m2, _, _ = api.pd_pack_delta(w_hat, L.d_w_b)
+    torch.cuda.synchronize()
+    moved = bits(host(w_hat)) != bits(L.w_b)
+    b1, b2 = orc.unpack(L.mask, 1024), orc.unpack(host(m2), 1024)
+    assert np.array_equal(b1[moved], b2[moved])
+
+
+# ------------------------------------------------------------------ decode linear
+def check_linear(api, L, m, axis, seed=2000, ldx_pad=0):
+    x = synth.gen_x(m, L.d_in, seed)
+    ref = orc.linear(x, L.w_b, L.mask, L.v(axis), axis)
+    d_x = dev(x)
+    if ldx_pad:
+        buf = torch.zeros((m, L.d_in + ldx_pad), dtype=torch.float16, device="cuda")
+        buf[:, :L.d_in] = d_x
+        d_x = buf[:, :L.d_in]
+    y = api.pd_linear(d_x, L.d_w_b, L.d_mask, L.d_v(axis), axis)
+    y2 = api.pd_linear(d_x, L.d_w_b, L.d_mask, L.d_v(axis), axis)
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == 0
+    err = rel_err(host(y), ref)
+    assert err <= TOL, (L.d_out, L.d_in, m, axis, err)
+    assert torch.equal(y, y2), "two runs must be bit-identical"
+    return err
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("m", [1, 16])
+def test_linear_config1(api, m, axis):
+    check_linear(api, layer(1024, 1024), m, axis)
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in,m", [(200, 1152, 3), (130, 384, 8), (65, 128, 9), (129, 2304, 16), (8, 128, 1),
+                                          (1000, 4224, 5), (64, 96, 7), (33, 1056, 16), (300, 32, 2)])
+def test_linear_ragged_shapes(api, d_out, d_in, m, axis):
+    check_linear(api, layer(d_out, d_in, seed=3), m, axis, ldx_pad=8 if m % 2 else 0)
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_linear_7b_decode(api, d_out, d_in, axis):
+    L = layer(d_out, d_in)
+    for m in (1, 4, 16):
+        check_linear(api, L, m, axis)
+
+
+def test_linear_sign_expansion_is_exact(api):
+    # W_b = 0, v = 1, small integer x: y = x . B^T is an exact integer, any bit-order slip shows
+    rng = np.random.default_rng(8)
+    d_out, d_in, m = 136, 640, 16
+    w_b = np.zeros((d_out, d_in), dtype=np.float16)
+    w_f = rng.choice([-1.0, 1.0], size=(d_out, d_in)).astype(np.float16)
+    mask, _, _ = orc.pack(w_f, w_b)
+    x = rng.integers(-3, 4, size=(m, d_in)).astype(np.float16)
+    ref = x.astype(np.float64) @ w_f.astype(np.float64).T
+    for axis, n in ((ROW, d_out), (COL, d_in)):
+        y = api.pd_linear(dev(x), dev(w_b), dev(mask), dev(np.ones(n, dtype=np.float16)), axis)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(y).astype(np.float64), ref)
+
+
+def test_linear_base_only_and_one_hot(api):
+    L = layer(1024, 1024)
+    x = synth.gen_x(4, 1024, 7)
+    y = api.pd_linear(dev(x), L.d_w_b, None, None, ROW)
+    torch.cuda.synchronize()
+    ref = x.astype(np.float64) @ L.w_b.astype(np.float64).T
+    assert rel_err(host(y), ref) <= TOL
+    # one-hot rows pick out columns of the merged weights exactly (one product, one fp32 add, RN16)
+    cols = [0, 1, 31, 32, 517, 1023]
+    xo = np.zeros((len(cols), 1024), dtype=np.float16)
+    xo[np.arange(len(cols)), cols] = 1.0
+    for axis in (ROW, COL):
+        y = api.pd_linear(dev(xo), L.d_w_b, L.d_mask, L.d_v(axis), axis)
+        torch.cuda.synchronize()
+        merged = orc.merge(L.w_b, L.mask, L.v(axis), axis)
+        assert np.array_equal(bits(host(y)), bits(merged[:, cols].T))
+
+
+@pytest.mark.parametrize("m", [17, 33, 40])
+def test_linear_between_decode_and_prefill(api, m):
+    check_linear(api, layer(1024, 1024), m, ROW)
+    check_linear(api, layer(200, 1152, seed=3), m, COL)
+
+
+# ------------------------------------------------------------------ multi-variant
+def make_variants(w_b, n_var, seed, mixed_axes=True, axis=ROW):
+    d_out, d_in = w_b.shape
+    masks = np.empty((n_var, d_out, d_in // 32), dtype=np.uint32)
+    stride = (max(d_out, d_in) + 7) // 8 * 8  # each variant's scales must start 16-byte aligned
+    vs = np.zeros((n_var, stride), dtype=np.float16)
+    axes = np.zeros(n_var, dtype=np.uint8)
+    for g in range(n_var):
+        w_f = synth.gen_finetuned(w_b, 1000 + seed + g)
+        m, vr, vc = orc.pack(w_f, w_b)
+        masks[g] = m
+        axes[g] = (g % 2) if mixed_axes else axis
+        if axes[g] == ROW:
+            vs[g, :d_out] = vr
+        else:
+            vs[g, :d_in] = vc
+    return masks, vs, axes
+
+
+@pytest.mark.parametrize("d_out,d_in,n_var,m", [(256, 512, 3, 20), (200, 1152, 4, 37), (130, 96, 2, 9), (1024, 1024, 16, 64)])
+def test_multivariant_small(api, d_out, d_in, n_var, m):
+    w_b = synth.gen_base(d_out, d_in, 11)
+    masks, vs, axes = make_variants(w_b, n_var, 11)
+    x = synth.gen_x(m, d_in, 12)
+    ids = synth.gen_ids(m, n_var, 13)
+    ids[1] = -1
+    ids[m - 1] = -1
+    ref, bad = orc.linear_multivariant(x, ids, w_b, masks, vs, axes)
+    assert bad == 0
+    args = (dev(x), dev(ids), dev(w_b), dev(masks), dev(vs), axes)
+    y = api.pd_linear_multivariant(*args)
+    y2 = api.pd_linear_multivariant(*args)
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == 0
+    assert rel_err(host(y), ref) <= TOL
+    assert torch.equal(y, y2)
+    # per-row check too: no row may borrow another variant's delta
+    yh = host(y).astype(np.float64)
+    for r in range(m):
+        assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
+
+
+def test_multivariant_bad_id_is_latched(api):
+    w_b = synth.gen_base(128, 128, 14)
+    masks, vs, axes = make_variants(w_b, 2, 14)
+    x = synth.gen_x(6, 128, 15)
+    ids = np.array([0, 1, 5, 0, -1, 1], dtype=np.int32)
+    y = api.pd_linear_multivariant(dev(x), dev(ids), dev(w_b), dev(masks), dev(vs), axes)
+    assert api.pd_device_status() == 6  # PD_ERR_BAD_VARIANT
+    assert api.pd_device_status() == 0  # cleared by the read
+    ref, bad = orc.linear_multivariant(x, ids, w_b, masks, vs, axes)
+    assert bad == 1
+    keep = [0, 1, 3, 4, 5]
+    assert rel_err(host(y)[keep], ref[keep]) <= TOL
+
+
+def test_native_library_is_the_one_in_tree(api):
+    import os
+    assert os.path.basename(api.LIB_PATH) == "libpd.so" and os.path.exists(api.LIB_PATH)
+    before = api.launch_count()
+    L = layer(1024, 1024)
+    api.pd_merge(L.d_w_b, L.d_mask, L.d_v_row, ROW)
+    torch.cuda.synchronize()
+    assert api.launch_count() == before + 1
