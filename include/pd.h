@@ -17,7 +17,9 @@
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
  *     The library never allocates or frees device memory and keeps no pointer after a call
  *     returns.  Scratch space comes from the caller through (workspace, workspace_bytes);
- *     pd_workspace_bytes() tells how much a call needs.  The workspace must be 256-byte aligned.
+ *     pd_workspace_bytes() tells how much a call needs.  The workspace must be 256-byte aligned,
+ *     and its first 256 bytes (the device status words) must be zero when it is first handed to
+ *     the library: zero-fill it once after allocating it.  pd_device_status() re-zeroes them.
  *   - cuda_stream is a cudaStream_t passed as void* (NULL = the legacy default stream).  Every
  *     call only enqueues work on that stream and returns without synchronising.
  *   - Errors that can be seen on the host (NULL pointers, bad sizes, misalignment, a short

@@ -8,6 +8,7 @@ namespace pd {
 namespace {
 
 constexpr int kMaxVariants = 64;
+constexpr int kGemvMaxTokens = 64;  // up to here the decode kernel runs in chunks of 16 rows
 constexpr int kGroupThreads = 1024;
 
 // workspace layout of the linear calls:
@@ -147,6 +148,9 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const __half *xh = static_cast<const __half *>(x);
     __half *yh = static_cast<__half *>(y);
+    if (M > kGemvMaxTokens)
+        return launch_gemm(xh, M, ldx, static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis,
+                           d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), stream);
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
         const int rows = static_cast<int>(M - m0 < 16 ? M - m0 : 16);
         st = launch_gemv(xh + m0 * ldx, rows, ldx, static_cast<const __half *>(w_b), mask,
@@ -178,7 +182,6 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
     auto *status = reinterpret_cast<uint32_t *>(base);
     int *offsets = reinterpret_cast<int *>(base + kStatusBytes);
     int *row_index = reinterpret_cast<int *>(base + kStatusBytes + kOffsetsBytes);
-    if (cudaMemsetAsync(status, 0, kStatusBytes, stream) != cudaSuccess) return PD_ERR_CUDA;
     st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, stream);
     if (st != PD_OK) return st;
     const __half *xh = static_cast<const __half *>(x);

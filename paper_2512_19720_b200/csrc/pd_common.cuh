@@ -41,6 +41,11 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
                       const int *row_index, const int *group_offsets, int group, cudaStream_t stream);
 
+// M > 16 tokens on the tcgen05 tensor cores (needs d_in % 8 == 0; tails in M, d_out and d_in are handled).
+pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
+                      const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
+                      uint32_t *status, cudaStream_t stream);
+
 // Stable bucket sort of token rows by variant id: offsets[g] .. offsets[g+1] index row_index for
 // variant g (g = 0..V-1), offsets[V] .. offsets[V+1] the rows with id -1.  Other ids latch an error.
 pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,

@@ -1,0 +1,448 @@
+// Prefill path: Y[M, d_out] = X . (W_b + v (.) B)^T on the 5th-generation tensor cores.
+//
+// The MMA computes the transposed tile  D[128 output rows, BN tokens] = W_hat_tile . X_tile^T :
+//   A operand = W_hat tile, 128 rows x 64 k, K-major, 128-byte swizzle, in shared memory
+//   B operand = X tile, BN tokens x 64 k, K-major, 128-byte swizzle, in shared memory
+//   D         = fp32 accumulator in tensor memory (two buffers, so the epilogue of one
+//               tile overlaps the main loop of the next)
+// Putting the weights on the 128-row side means each W_b tile is expanded once per BN = 256
+// tokens, the largest reuse one CTA can get.
+//
+// Pipeline per 64-wide k step (4 smem stages):
+//   producer warp   : TMA loads of the W_b tile and the X tile -> full[s]
+//   transform warps : wait full[s]; read the W_b tile from shared memory, add +-v per element
+//                     according to the mask word fetched from global memory, write it back in
+//                     place (same swizzled position), fence for the async proxy -> xform[s]
+//   MMA warp        : wait xform[s]; four tcgen05.mma (K = 16 each); commit -> empty[s]
+//   epilogue warps  : wait acc_full[b]; tcgen05.ld the 32 lanes they own, convert to fp16 and
+//                     store y[token][row]; -> acc_empty[b]
+// Every wait is bounded; a wait that runs out latches PD_ERR_DEVICE_TIMEOUT and the CTA
+// drains and exits.
+#include <cuda.h>
+
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+constexpr int BM = 128;          // output rows per tile (MMA M)
+constexpr int BK = 64;           // k per stage: 128 bytes of fp16 = one swizzle atom
+constexpr int kStages = 4;
+constexpr int kAccCols = 256;    // TMEM columns per accumulator buffer
+constexpr int kNumWarps = 14;    // 0 producer, 1 MMA, 2-5 epilogue, 6-13 transform
+constexpr int kNumThreads = kNumWarps * 32;
+constexpr int kXformWarps = 8;
+constexpr int kEpiWarps = 4;
+constexpr long long kWaitCycles = 2000000000ll;  // ~1 s: far beyond any legitimate wait
+
+struct GemmArgs {
+    const uint32_t *mask;  // [d_out, d_in/32] or nullptr (base only)
+    const __half *v;
+    __half *y;
+    int64_t ldy;
+    int M, d_out, d_in;
+    int tiles_m, tiles_n, k_steps;
+    uint32_t *status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                          uint32_t where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                latch_error(status, PD_ERR_DEVICE_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap *map, uint64_t *bar, void *dst, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_alloc(uint32_t *dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// (~a & b) ^ c
+__device__ __forceinline__ uint32_t lop3_andn_xor(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xA6;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t hadd2_u32(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
+// 1024 bytes apart; `addr` is the byte address of the first row (plus the k offset inside the atom).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                       // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                       // 128-byte swizzle
+    return d;
+}
+
+template <int BN>
+struct SmemLayout {
+    static constexpr int kWBytes = BM * BK * 2;   // 16 KB
+    static constexpr int kXBytes = BN * BK * 2;   // 32 KB for BN = 256
+    static constexpr int kStageBytes = kWBytes + kXBytes;
+    static constexpr int kBarOffset = kStages * kStageBytes;
+    static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+};
+
+template <int AXIS, bool HAS_DELTA, int BN>
+__global__ void __launch_bounds__(kNumThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
+    using L = SmemLayout<BN>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
+    uint64_t *full = bars, *xform = bars + kStages, *empty = bars + 2 * kStages;
+    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = bars + 3 * kStages + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * kStages + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = a.tiles_m * a.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(xform + s, kXformWarps);
+            mbar_init(empty + s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full + b, 1);
+            mbar_init(acc_empty + b, kEpiWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tcgen05_alloc(tmem_slot, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int tm = tile / a.tiles_n, tn = tile - tm * a.tiles_n;
+                for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
+                    const int s = it % kStages;
+                    if (!(ok = mbar_wait(empty + s, ((it / kStages) & 1) ^ 1, abort_flag, a.status, 1))) break;
+                    unsigned char *st = smem + s * L::kStageBytes;
+                    mbar_arrive_expect_tx(full + s, L::kStageBytes);
+                    tma_load_2d(&map_w, full + s, st, ks * BK, tm * BM);
+                    tma_load_2d(&map_x, full + s, st + L::kWBytes, ks * BK, tn * BN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+                const uint32_t b = tcount & 1;
+                if (!(ok = mbar_wait(acc_empty + b, ((tcount >> 1) & 1) ^ 1, abort_flag, a.status, 2))) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + b * kAccCols;
+                for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
+                    const int s = it % kStages;
+                    if (!(ok = mbar_wait(xform + s, (it / kStages) & 1, abort_flag, a.status, 3))) break;
+                    tcgen05_fence_after();
+                    const uint32_t w_addr = smem_u32(smem + s * L::kStageBytes);
+                    const uint32_t x_addr = w_addr + L::kWBytes;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        const uint64_t da = make_smem_desc(w_addr + kk * 32);
+                        const uint64_t db = make_smem_desc(x_addr + kk * 32);
+                        tcgen05_mma_f16(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tcgen05_commit(empty + s);  // frees the stage when these MMAs have read it
+                }
+                if (ok) tcgen05_commit(acc_full + b);
+            }
+        }
+    } else if (warp < 2 + kEpiWarps) {
+        // ------------------------------------------------ epilogue: TMEM -> fp16 -> y[token][row]
+        const int quarter = warp & 3;  // the 32 TMEM lanes this warp may read
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+            const int tm = tile / a.tiles_n, tn = tile - tm * a.tiles_n;
+            const uint32_t b = tcount & 1;
+            if (!(ok = mbar_wait(acc_full + b, (tcount >> 1) & 1, abort_flag, a.status, 4))) break;
+            tcgen05_fence_after();
+            const int o = tm * BM + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * kAccCols;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tcgen05_ld_32x32b_x32(taddr + c0, r);
+                tcgen05_wait_ld();
+                const int tok0 = tn * BN + c0;
+                if (o < a.d_out) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (tok0 + j < a.M)
+                            a.y[static_cast<size_t>(tok0 + j) * a.ldy + o] = __float2half_rn(__uint_as_float(r[j]));
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty + b);
+        }
+    } else {
+        // ------------------------------------------------ transform: W_b tile -> W_hat tile, in place
+        const int tt = threadIdx.x - (2 + kEpiWarps) * 32;  // 0..255
+        const int r = tt >> 1, h = tt & 1;                   // tile row, 32-column half of the stage
+        const int words = a.d_in >> 5;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const int tm = tile / a.tiles_n;
+            const int o = tm * BM + r;
+            const bool row_ok = o < a.d_out;
+            uint32_t vrow = 0;
+            if (HAS_DELTA && AXIS == PD_AXIS_ROW && row_ok) {
+                const uint32_t hv = *reinterpret_cast<const unsigned short *>(a.v + o);
+                vrow = hv | (hv << 16);
+            }
+            const uint32_t *mrow = HAS_DELTA ? a.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
+            uint32_t word_next = 0;
+            if (HAS_DELTA && row_ok && h < words) word_next = __ldg(mrow + h);
+            for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
+                const int s = it % kStages;
+                const uint32_t word = word_next;
+                if (HAS_DELTA) {
+                    const int wi = 2 * (ks + 1) + h;
+                    word_next = (row_ok && ks + 1 < a.k_steps && wi < words) ? __ldg(mrow + wi) : 0u;
+                }
+                if (!(ok = mbar_wait(full + s, (it / kStages) & 1, abort_flag, a.status, 5))) break;
+                if (HAS_DELTA) {
+                    unsigned char *wt = smem + s * L::kStageBytes + r * 128;
+                    uint32_t sh[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) sh[q] = word << q;  // bit 8j+q' on top of byte j in sh[7-q']
+                    const int kcol = ks * BK + 32 * h;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 *p = reinterpret_cast<uint4 *>(wt + ((((4 * h + j) ^ (r & 7))) << 4));
+                        uint4 w = *p;
+                        uint32_t vv[4] = {vrow, vrow, vrow, vrow};
+                        if (AXIS == PD_AXIS_COL) {
+                            const int k = kcol + 8 * j;
+                            uint4 t4 = make_uint4(0, 0, 0, 0);
+                            if (k < a.d_in) t4 = __ldg(reinterpret_cast<const uint4 *>(a.v + k));
+                            vv[0] = t4.x; vv[1] = t4.y; vv[2] = t4.z; vv[3] = t4.w;
+                        }
+                        const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
+                        uint32_t *wp = reinterpret_cast<uint32_t *>(&w);
+#pragma unroll
+                        for (int pr = 0; pr < 4; ++pr) {
+                            // halves 2pr (low) and 2pr+1 (high) of this 8-column piece: +v where the bit is 1, -v where 0
+                            const uint32_t rep = prmt(sh[7 - 2 * pr], sh[6 - 2 * pr], sel);
+                            wp[pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
+                        }
+                        *p = w;
+                    }
+                    fence_proxy_async_smem();
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(xform + s);
+            }
+        }
+    }
+
+    // ------------------------------------------------ teardown
+    tcgen05_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait ran out somewhere: give copies that may still be in flight time to land
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        tcgen05_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeFn>(p);
+    }();
+    return fn;
+}
+
+// fp16 row-major [rows, cols] with row pitch ld elements; box = 64 columns x box_rows rows, 128-byte swizzle
+bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[2] = {BK, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int AXIS, bool HAS_DELTA, int BN>
+pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    auto kernel = gemm_kernel<AXIS, HAS_DELTA, BN>;
+    constexpr int smem = SmemLayout<BN>::kTotal;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return PD_ERR_CUDA;
+        configured = true;
+    }
+    kernel<<<grid, kNumThreads, smem, stream>>>(mw, mx, args);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        return v;
+    }();
+    return n;
+}
+
+}  // namespace
+
+pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
+                      const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
+                      uint32_t *status, cudaStream_t stream) {
+    constexpr int BN = 256;
+    CUtensorMap mw, mx;
+    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, BN)) return PD_ERR_CUDA;
+    GemmArgs args;
+    args.mask = mask;
+    args.v = v;
+    args.y = y;
+    args.ldy = ldy;
+    args.M = static_cast<int>(M);
+    args.d_out = static_cast<int>(d_out);
+    args.d_in = static_cast<int>(d_in);
+    args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
+    args.tiles_n = static_cast<int>((M + BN - 1) / BN);
+    args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
+    args.status = status;
+    const int tiles = args.tiles_m * args.tiles_n;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    if (mask == nullptr) return launch_one<PD_AXIS_ROW, false, BN>(mw, mx, args, grid, stream);
+    if (axis == PD_AXIS_ROW) return launch_one<PD_AXIS_ROW, true, BN>(mw, mx, args, grid, stream);
+    return launch_one<PD_AXIS_COL, true, BN>(mw, mx, args, grid, stream);
+}
+
+}  // namespace pd

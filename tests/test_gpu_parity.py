@@ -234,6 +234,65 @@ def test_linear_between_decode_and_prefill(api, m):
     check_linear(api, layer(200, 1152, seed=3), m, COL)
 
 
+# ------------------------------------------------------------------ prefill linear (tensor-core path)
+def check_prefill(api, L, m, axis, rows=None, seed=2000):
+    x = synth.gen_x(m, L.d_in, seed)
+    y = api.pd_linear(dev(x), L.d_w_b, L.d_mask, L.d_v(axis), axis)
+    y2 = api.pd_linear(dev(x), L.d_w_b, L.d_mask, L.d_v(axis), axis)
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == 0
+    assert torch.equal(y, y2)
+    yh = host(y)
+    if rows is None:
+        ref = orc.linear(x, L.w_b, L.mask, L.v(axis), axis)
+        err = rel_err(yh, ref)
+    else:
+        ref = orc.linear(np.ascontiguousarray(x[rows]), L.w_b, L.mask, L.v(axis), axis)
+        err = rel_err(yh[rows], ref)
+        assert np.isfinite(yh.astype(np.float32)).all()
+    assert err <= TOL, (L.d_out, L.d_in, m, axis, err)
+    return err
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in,m", [(1024, 1024, 256), (128, 64, 65), (200, 1152, 100), (130, 96, 257),
+                                          (1000, 4224, 300), (64, 32, 70), (129, 2304, 513), (256, 512, 1024)])
+def test_prefill_small_shapes(api, d_out, d_in, m, axis):
+    check_prefill(api, layer(d_out, d_in, seed=3 if d_out != 1024 else 0), m, axis)
+
+
+def test_prefill_base_only_and_exact_signs(api):
+    L = layer(1024, 1024)
+    x = synth.gen_x(300, 1024, 7)
+    y = api.pd_linear(dev(x), L.d_w_b, None, None, ROW)
+    torch.cuda.synchronize()
+    assert rel_err(host(y), x.astype(np.float64) @ L.w_b.astype(np.float64).T) <= TOL
+    # W_b = 0, v = 1: W_hat = B exactly, small-integer x gives exact integer outputs
+    rng = np.random.default_rng(9)
+    d_out, d_in, m = 200, 320, 130
+    w_b = np.zeros((d_out, d_in), dtype=np.float16)
+    w_f = rng.choice([-1.0, 1.0], size=(d_out, d_in)).astype(np.float16)
+    mask, _, _ = orc.pack(w_f, w_b)
+    xi = rng.integers(-3, 4, size=(m, d_in)).astype(np.float16)
+    ref = xi.astype(np.float64) @ w_f.astype(np.float64).T
+    for axis, n in ((ROW, d_out), (COL, d_in)):
+        y = api.pd_linear(dev(xi), dev(w_b), dev(mask), dev(np.ones(n, dtype=np.float16)), axis)
+        torch.cuda.synchronize()
+        assert api.pd_device_status() == 0
+        assert np.array_equal(host(y).astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+def test_prefill_7b_m256_full(api, axis):
+    check_prefill(api, layer(4096, 4096), 256, axis)
+
+
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in,m", [(4096, 4096, 2048), (11008, 4096, 2048), (4096, 11008, 2048), (4096, 4096, 8192)])
+def test_prefill_7b_sampled_rows(api, d_out, d_in, m, axis):
+    check_prefill(api, layer(d_out, d_in), m, axis, rows=synth.sample_rows(m, n_random=16))
+
+
 # ------------------------------------------------------------------ multi-variant
 def make_variants(w_b, n_var, seed, mixed_axes=True, axis=ROW):
     d_out, d_in = w_b.shape
