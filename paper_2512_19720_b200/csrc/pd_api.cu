@@ -148,7 +148,7 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const __half *xh = static_cast<const __half *>(x);
     __half *yh = static_cast<__half *>(y);
-    if (M > kGemvMaxTokens)
+    if (M > kGemvMaxTokens && d_in >= 64)  // narrower layers would need a TMA box wider than the matrix
         return launch_gemm(xh, M, ldx, static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis,
                            d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), stream);
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
