@@ -134,6 +134,32 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
 pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
                    int64_t d_out, int64_t d_in, void *w_hat, void *cuda_stream);
 
+/*
+ * pd_pack_delta_static -- pd_pack_delta without a workspace argument and without any allocation.
+ * The paper has no counterpart: this entry point exists for the library's users, not the method.
+ *
+ * Some callers have no way to obtain scratch memory at the point where they pack a layer: code
+ * that runs inside a memory pool whose budget is already fixed, a plug-in that is handed tensors
+ * by a host framework but must not call the CUDA allocator (cudaMalloc synchronises the device
+ * and is forbidden while a stream is being captured), or a C program that links no allocator
+ * wrapper at all.  For them the exact per-row and per-column sums of |dW| are kept in a fixed
+ * 512 KiB array that is part of the library's device image (one copy on every GPU that loads the
+ * library, held until the process exits).
+ *
+ *   arguments : as pd_pack_delta, minus (workspace, workspace_bytes); results are bit-identical.
+ *   limit     : d_out + d_in <= 65536, else PD_ERR_UNSUPPORTED_SHAPE (nothing is launched).
+ *   set-up    : the first call on each device looks up the array's device address (the device
+ *               must be current, as for every call).  Make that first call outside any stream
+ *               capture.
+ *   sharing   : all calls on one GPU use the same array.  Each call zero-fills the part it uses
+ *               on its stream first, so back-to-back calls on ONE stream are safe; calls that may
+ *               overlap on the GPU (different streams, different threads) race on it and give
+ *               wrong scales -- serialise them or use pd_pack_delta with separate workspaces.
+ *   It calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+pd_status pd_pack_delta_static(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in,
+                               uint32_t *mask, void *v_row, void *v_col, void *cuda_stream);
+
 /* Bytes of workspace the given call needs (0 for PD_OP_MERGE).  M and V are ignored where they
  * do not apply.  Returns 0 for an unknown op. */
 size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d_in);

@@ -18,7 +18,7 @@ OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE = 0, 1, 2, 3
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpd.so")
 
-EXPORTS = ["pd_pack_delta", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
+EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
            "pd_device_status", "pd_status_string", "pd_launch_count"]
 
 
@@ -36,6 +36,8 @@ def _load() -> ctypes.CDLL:
     p, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
     lib.pd_pack_delta.argtypes = [p, p, i64, i64, p, p, p, p, sz, p]
     lib.pd_pack_delta.restype = ctypes.c_int
+    lib.pd_pack_delta_static.argtypes = [p, p, i64, i64, p, p, p, p]
+    lib.pd_pack_delta_static.restype = ctypes.c_int
     lib.pd_linear.argtypes = [p, i64, i64, p, p, p, ctypes.c_int, i64, i64, p, i64, p, sz, p]
     lib.pd_linear.restype = ctypes.c_int
     lib.pd_linear_multivariant.argtypes = [p, i64, i64, p, p, p, p, i64, p, i32, i64, i64, p, i64, p, sz, p]
@@ -117,6 +119,19 @@ def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None,
                              _ptr(v_col if want_col else None), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "pd_pack_delta")
     return mask, (v_row if want_row else None), (v_col if want_col else None)
+
+
+def pd_pack_delta_static(w_f, w_b, mask, v_row=None, v_col=None):
+    """pd_pack_delta for callers that cannot allocate: every output is a tensor the caller already
+    owns, the scratch sums live in a fixed array inside the library (d_out + d_in <= 65536), and
+    neither this wrapper nor the library call allocates anything.  Calls that overlap on one GPU
+    race on that array; calls queued on one stream do not."""
+    _want(w_f, torch.float16, "w_f"), _want(w_b, torch.float16, "w_b")
+    assert w_f.shape == w_b.shape and w_f.is_contiguous() and w_b.is_contiguous()
+    d_out, d_in = w_b.shape
+    _check(lib.pd_pack_delta_static(_ptr(w_f), _ptr(w_b), d_out, d_in, _ptr(mask), _ptr(v_row), _ptr(v_col),
+                                    _stream()), "pd_pack_delta_static")
+    return mask, v_row, v_col
 
 
 def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None):

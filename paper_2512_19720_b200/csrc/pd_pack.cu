@@ -254,3 +254,51 @@ pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v,
 }
 
 }  // namespace pd
+
+// ---------------------------------------------------------------------------------------------
+// pd_pack_delta_static: the pack call for callers that cannot hand over a workspace.
+//
+// The exact sums of |dW| (one 64-bit word per output row and per input column) live in the
+// file-scope device array below instead of in caller memory.  The array is part of the loaded
+// module: every GPU that loads the library carries its 512 KiB until the process exits.
+// In host code `g_static_sums` is only a handle; the device address comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+namespace pd {
+namespace {
+
+constexpr int64_t kStaticSumWords = 65536;  // d_out + d_in may not exceed this
+static __device__ __align__(256) unsigned long long g_static_sums[kStaticSumWords];
+
+constexpr int kMaxDevices = 64;
+std::atomic<unsigned long long *> g_static_sums_addr[kMaxDevices];
+
+// Device address of g_static_sums on the current device (nullptr on failure).
+unsigned long long *static_sums_on_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    unsigned long long *p = g_static_sums_addr[dev].load(std::memory_order_acquire);
+    if (p != nullptr) return p;
+    void *sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_static_sums) != cudaSuccess || sym == nullptr) return nullptr;
+    p = static_cast<unsigned long long *>(sym);
+    g_static_sums_addr[dev].store(p, std::memory_order_release);  // every thread resolves the same address
+    return p;
+}
+
+}  // namespace
+}  // namespace pd
+
+extern "C" pd_status pd_pack_delta_static(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in,
+                                          uint32_t *mask, void *v_row, void *v_col, void *cuda_stream) {
+    using namespace pd;
+    if (!w_f || !w_b || !mask || (!v_row && !v_col) || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || d_out > kStaticSumWords || d_in > kStaticSumWords || d_out + d_in > kStaticSumWords)
+        return PD_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(w_f) || !aligned16(w_b) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
+    unsigned long long *sums = static_sums_on_current_device();
+    if (sums == nullptr) return PD_ERR_CUDA;
+    // launch_pack zero-fills sums[0 .. d_out + d_in) on the stream before the kernel adds into it
+    return launch_pack(static_cast<const __half *>(w_f), static_cast<const __half *>(w_b), d_out, d_in, mask,
+                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
