@@ -151,11 +151,13 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
     if (M > kGemvMaxTokens && d_in >= 64)  // narrower layers would need a TMA box wider than the matrix
         return launch_gemm(xh, M, ldx, static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis,
                            d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), stream);
+    GemvScratch scratch;
+    scratch.status = static_cast<uint32_t *>(workspace);
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
         const int rows = static_cast<int>(M - m0 < 16 ? M - m0 : 16);
         st = launch_gemv(xh + m0 * ldx, rows, ldx, static_cast<const __half *>(w_b), mask,
                          static_cast<const __half *>(v), axis, d_out, d_in, yh + m0 * ldy, ldy, nullptr, nullptr, 0,
-                         stream);
+                         &scratch, stream);
         if (st != PD_OK) return st;
     }
     return PD_OK;
@@ -191,7 +193,7 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
         const bool base_only = (g == V);
         st = launch_gemv(xh, 0, ldx, static_cast<const __half *>(w_b), base_only ? nullptr : masks + g * mask_words,
                          base_only ? nullptr : vh + g * v_stride, base_only ? PD_AXIS_ROW : axes[g], d_out, d_in,
-                         static_cast<__half *>(y), ldy, row_index, offsets, g, stream);
+                         static_cast<__half *>(y), ldy, row_index, offsets, g, nullptr, stream);
         if (st != PD_OK) return st;
     }
     return PD_OK;

@@ -35,11 +35,18 @@ pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64
 pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
                        int64_t d_in, __half *w_hat, cudaStream_t stream);
 
+// What the decode kernels need from the caller's workspace.
+struct GemvScratch {
+    uint32_t *status;  // device status words
+};
+
 // M <= 16 tokens (mask == nullptr: base weights only).  With group_offsets != nullptr the tokens are
 // rows row_index[group_offsets[group] .. group_offsets[group+1]) of x / y (any count, read on the device).
+// scratch may be nullptr (then the register-fed kernel runs); it is required for nothing else.
 pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      const int *row_index, const int *group_offsets, int group, cudaStream_t stream);
+                      const int *row_index, const int *group_offsets, int group, const GemvScratch *scratch,
+                      cudaStream_t stream);
 
 // M > 16 tokens on the tcgen05 tensor cores (needs d_in % 8 == 0; tails in M, d_out and d_in are handled).
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,

@@ -18,7 +18,7 @@
 
 #include <cstdlib>
 
-#include "pd_common.cuh"
+#include "pd_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -39,19 +39,6 @@ __device__ __forceinline__ uint4 ldg_stream(const void *p) {
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                  : "l"(p));
     return r;
-}
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// (~a & b) | c
-__device__ __forceinline__ uint32_t lop3_nand_or(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xAE;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
 }
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -211,7 +198,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
                         uint32_t pm[4];
 #pragma unroll
                         for (int r = 0; r < 4; ++r)
-                            pm[r] = lop3_nand_or(prmt(sh[j][7 - 2 * r], sh[j][6 - 2 * r], sel), 0x80008000u, 0x3C003C00u);
+                            pm[r] = lop3_andn_or(prmt(sh[j][7 - 2 * r], sh[j][6 - 2 * r], sel), 0x80008000u, 0x3C003C00u);
                         mma16816(acc_d[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
                         mma16816(acc_d[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
                     }
@@ -248,6 +235,219 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
     }
     cluster.sync();  // keep shared memory alive until every rank has read it
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Streaming decode kernel: weights brought in by TMA, one CTA per 32 output rows, two CTAs per SM.
+//
+// A CTA owns 32 rows for the whole of d_in, so its result needs no other CTA: no partial sums in
+// global memory, no tickets, no fences.  It walks d_in in steps of 256 columns; a step is 16 KB of
+// W_b (one TMA box of four 64-column blocks, 128-byte swizzle), 1 KB of mask, the matching 256
+// columns of x and, for the col axis, of v: four TMA instructions per step.  One producer lane keeps
+// a ring of four steps in flight (64 KB of weights per CTA, 128 KB per SM), so an SM's whole share of
+// a 7B-sized layer is requested within the first microsecond.  Fewer CTAs than SMs (4096 rows = 128
+// CTAs) is fine: HBM, not the SM count, is the limit, and an SM with deep queues can pull well above
+// its fair share.
+//
+// Eight consumer warps: warp pair p takes the steps s = p (mod 4), which always sit in stage p, so a
+// warp sees every phase of the barriers it waits on in order; inside a pair each warp takes two of
+// the four column blocks and all 32 rows (four n8 tiles), so an x fragment read from shared memory
+// feeds four tiles.  16-byte pieces are read conflict free from the swizzled tiles: lane (g,t)
+// takes pieces t and t+4 of row g of a block.  The eight partial accumulators are added in warp order
+// through shared memory (the buffer reuses the drained ring).
+//
+// Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the
+// stream, so their loads are issued before griddepcontrol.wait; x is loaded and y stored after it.
+constexpr int kStreamRows = 32;
+constexpr int kStreamK = 256;
+constexpr int kStreamStages = 4;
+constexpr int kStreamConsumers = 8;
+constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
+constexpr int kStW = 0;                     // [32 rows][4 blocks][128 B], swizzled
+constexpr int kStX = 16384;                 // [16 rows][4 blocks][128 B], swizzled
+constexpr int kStMask = kStX + 8192;        // [32 rows][8 words]
+constexpr int kStV = kStMask + 1024;        // 256 fp16 (col axis)
+constexpr int kStageBytes = 26 * 1024;      // rounded up: every stage starts 1024-byte aligned
+constexpr int kRedOffset = 0;               // [8 warps][16 tokens][32 rows] fp32, over the ring once it has drained
+constexpr int kBarOffset = kStreamStages * kStageBytes;
+constexpr int kStreamSmem = kBarOffset + 256 + 1024 /* alignment slack */;
+static_assert(kStreamStages == 4, "stage p belongs to warp pair p");
+static_assert(kStreamConsumers * 16 * kStreamRows * 4 <= kStreamStages * kStageBytes, "reduction buffer must fit the ring");
+
+struct StreamArgs {
+    const __half *v;
+    __half *y;
+    int64_t ldy;
+    int M, d_out, d_in;
+    int n_k;  // steps of 256 columns (the last one may be half empty)
+    uint32_t *status;
+};
+
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+template <int AXIS, bool HAS_DELTA, bool M16>
+__global__ void __maxnreg__(112)
+gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                   const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    float *red = reinterpret_cast<float *>(smem + kRedOffset);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + kBarOffset);
+    uint64_t *empty = full + kStreamStages;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + kStreamStages);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = blockIdx.x * kStreamRows;
+    constexpr bool kCol = HAS_DELTA && AXIS == PD_AXIS_COL;
+    constexpr uint32_t kWBytes = 16384u + (HAS_DELTA ? 1024u : 0u);
+    constexpr uint32_t kXBytes = M16 ? 8192u : 4096u;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStreamStages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, 2);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == kStreamConsumers) {
+        // ------------------------------------------------ producer
+        if (lane == 0) {
+            grid_launch_dependents();  // the next kernel in the stream may start its own weight loads
+            // bytes of v in step s (the last step of a d_in that is not a multiple of 256 has 128 columns)
+            auto v_bytes = [&](int s) { return static_cast<uint32_t>(min(kStreamK, a.d_in - s * kStreamK) * 2); };
+            auto load_w = [&](int s, int st) {
+                unsigned char *base = smem + st * kStageBytes;
+                tma_load_3d(&map_w, full + st, base + kStW, 0, s * 4, row0);
+                if (HAS_DELTA) tma_load_2d(&map_m, full + st, base + kStMask, s * 8, row0);
+                if (kCol) bulk_load_1d(base + kStV, a.v + static_cast<size_t>(s) * kStreamK, v_bytes(s), full + st);
+            };
+            auto load_x = [&](int s, int st) { tma_load_3d(&map_x, full + st, smem + st * kStageBytes + kStX, 0, s * 4, 0); };
+            const int pre = min(a.n_k, kStreamStages);
+            for (int s = 0; s < pre; ++s) {  // weights first: they do not depend on earlier work in the stream
+                mbar_expect_tx(full + s, kWBytes + (kCol ? v_bytes(s) : 0u));
+                load_w(s, s);
+            }
+            grid_dependency_wait();  // x may be the previous kernel's output
+            for (int s = 0; s < pre; ++s) {
+                mbar_arrive_expect_tx(full + s, kXBytes);
+                load_x(s, s);
+            }
+            for (int s = pre; s < a.n_k; ++s) {
+                const int st = s % kStreamStages;
+                if (!mbar_wait(empty + st, ((s / kStreamStages) & 1) ^ 1, abort_flag, a.status, 11)) break;
+                mbar_arrive_expect_tx(full + st, kWBytes + kXBytes + (kCol ? v_bytes(s) : 0u));
+                load_w(s, st);
+                load_x(s, st);
+            }
+        }
+    } else {
+        // ------------------------------------------------ consumers
+        const int g = lane >> 2, t = lane & 3;
+        const int pair = warp >> 1, half = warp & 1;  // stage / steps of this pair; which two column blocks
+        const uint32_t sel_t = static_cast<uint32_t>(t | ((4 + t) << 4));
+        // One accumulator per tile: the delta term enters as x . (+-s) with s = v[row] (row axis, exact
+        // fp16 products summed in fp32) or as (x*v) . (+-1) (col axis).
+        float acc[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
+        uint32_t mag[4];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            mag[j] = 0x3C003C00u;
+            if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
+                const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
+                mag[j] = h | (h << 16);
+            }
+        }
+        bool ok = true;
+        const unsigned char *base = smem + pair * kStageBytes;
+        for (int s = pair; s < a.n_k; s += 4) {
+            if (!(ok = mbar_wait(full + pair, (s / kStreamStages) & 1, abort_flag, a.status, 12))) break;
+            uint32_t my[4];  // per tile: byte 2*b + c = sign bits of piece t + 4c of this warp's block b
+            if (HAS_DELTA) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 m = *reinterpret_cast<const uint4 *>(base + kStMask + (8 * j + g) * 32 + half * 16);
+                    my[j] = prmt(prmt(m.x, m.y, sel_t), prmt(m.z, m.w, sel_t), 0x5410u);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const int blk = 2 * half + b;
+                if (s * kStreamK + blk * 64 >= a.d_in) continue;  // past the end of d_in: nothing was loaded there
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    // byte offset inside a row of the box, swizzled: piece index ^ (bits 7..9 of the offset)
+                    const uint32_t piece = static_cast<uint32_t>(t + 4 * c);
+                    const uint32_t in_row = static_cast<uint32_t>(blk * 128) + ((piece ^ static_cast<uint32_t>(((g & 1) << 2) | blk)) << 4);
+                    const uint4 xa = *reinterpret_cast<const uint4 *>(base + kStX + g * 512 + in_row);
+                    uint4 xb = make_uint4(0, 0, 0, 0);
+                    if (M16) xb = *reinterpret_cast<const uint4 *>(base + kStX + (g + 8) * 512 + in_row);
+                    uint4 da = xa, db = xb;
+                    if (kCol) {
+                        const uint4 vv = *reinterpret_cast<const uint4 *>(base + kStV + blk * 128 + (piece << 4));
+                        da = make_uint4(hmul2_u32(xa.x, vv.x), hmul2_u32(xa.y, vv.y), hmul2_u32(xa.z, vv.z), hmul2_u32(xa.w, vv.w));
+                        if (M16) db = make_uint4(hmul2_u32(xb.x, vv.x), hmul2_u32(xb.y, vv.y), hmul2_u32(xb.z, vv.z), hmul2_u32(xb.w, vv.w));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 w = *reinterpret_cast<const uint4 *>(base + kStW + (8 * j + g) * 512 + in_row);
+                        mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                        mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                        if (HAS_DELTA) {
+                            // pair r = halves 2r, 2r+1 of the piece: bit 2r of byte i -> bit 15, bit 2r+1 -> bit 31;
+                            // a clear bit (B = -1) flips the sign of the magnitude
+                            const int i = 2 * b + c;
+                            const uint32_t sel = static_cast<uint32_t>(((i | 8) << 4) | (((4 + i) | 8) << 12));
+                            uint32_t pm[4];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r)
+                                pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mag[j]);
+                            mma16816(acc[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
+                            mma16816(acc[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + pair);
+        }
+
+        // ---- add the eight warps' partial sums in warp order (the buffer reuses the ring: every step
+        // has been consumed once all consumer warps are past this barrier)
+        asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
+        if (ok) {
+            float *mine = red + warp * 16 * kStreamRows;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int ol = 8 * j + 2 * t + e;
+                    mine[g * kStreamRows + ol] = acc[j][e];
+                    mine[(g + 8) * kStreamRows + ol] = acc[j][2 + e];
+                }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
+        if (!*abort_flag) {
+            grid_dependency_wait();
+            for (int idx = threadIdx.x; idx < 16 * kStreamRows; idx += kStreamConsumers * 32) {
+                const int tok = idx / kStreamRows, ol = idx - tok * kStreamRows;
+                float sum = 0.f;
+#pragma unroll
+                for (int w = 0; w < kStreamConsumers; ++w) sum += red[(w * 16 + tok) * kStreamRows + ol];
+                if (tok < a.M && row0 + ol < a.d_out) a.y[static_cast<size_t>(tok) * a.ldy + row0 + ol] = __float2half_rn(sum);
+            }
+        }
+    }
 }
 
 // Any d_in that is a multiple of 32 (the tensor path above needs a multiple of 128): one warp per
@@ -302,6 +502,11 @@ __global__ void __launch_bounds__(256) gemv_generic_kernel(const GemvArgs a) {
   }
 }
 
+int env_int(const char *name, int fallback) {
+    const char *s = getenv(name);
+    return s ? atoi(s) : fallback;
+}
+
 template <int AXIS, bool HAS_DELTA, bool M16>
 pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) {
     constexpr int tok = M16 ? 16 : 8;
@@ -331,16 +536,77 @@ pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) 
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, args));
 }
 
-int env_int(const char *name, int fallback) {
-    const char *s = getenv(name);
-    return s ? atoi(s) : fallback;
+template <int AXIS, bool HAS_DELTA, bool M16>
+pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mx, const CUtensorMap &mm, const StreamArgs &args,
+                                int grid, cudaStream_t stream) {
+    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16>;
+    static bool configured = false;  // per instantiation
+    if (!configured) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem) != cudaSuccess)
+            return PD_ERR_CUDA;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = kStreamSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may start while the previous kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static const int use_pdl = env_int("PD_PDL", 1);
+    cfg.numAttrs = use_pdl ? 1 : 0;
+    count_launch();
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, mm, args));
+}
+
+pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
+                        int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                        cudaStream_t stream) {
+    const bool m16 = M > 8, delta = mask != nullptr;
+    CUtensorMap mw, mx, mm;
+    if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, kStreamRows) ||
+        !make_map_blocked_f16(&mx, x, M, d_in, ldx * 2, 4, m16 ? 16 : 8))
+        return PD_ERR_CUDA;
+    mm = mw;
+    if (delta && !make_map_2d(&mm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, mask, d_out, d_in / 32, d_in / 8, 8, kStreamRows,
+                              CU_TENSOR_MAP_SWIZZLE_NONE))
+        return PD_ERR_CUDA;
+    StreamArgs a;
+    a.v = v;
+    a.y = y;
+    a.ldy = ldy;
+    a.M = M;
+    a.d_out = static_cast<int>(d_out);
+    a.d_in = static_cast<int>(d_in);
+    a.n_k = static_cast<int>((d_in + kStreamK - 1) / kStreamK);
+    a.status = status;
+    const int grid = static_cast<int>((d_out + kStreamRows - 1) / kStreamRows);
+#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W>(mw, mx, mm, a, grid, stream)
+    if (!delta) {
+        if (m16) PD_STREAM_CASE(PD_AXIS_ROW, false, true);
+        PD_STREAM_CASE(PD_AXIS_ROW, false, false);
+    }
+    if (axis == PD_AXIS_ROW) {
+        if (m16) PD_STREAM_CASE(PD_AXIS_ROW, true, true);
+        PD_STREAM_CASE(PD_AXIS_ROW, true, false);
+    }
+    if (m16) PD_STREAM_CASE(PD_AXIS_COL, true, true);
+    PD_STREAM_CASE(PD_AXIS_COL, true, false);
+#undef PD_STREAM_CASE
 }
 
 }  // namespace
 
 pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      const int *row_index, const int *group_offsets, int group, cudaStream_t stream) {
+                      const int *row_index, const int *group_offsets, int group, const GemvScratch *ws,
+                      cudaStream_t stream) {
+    // plain calls on TMA-friendly shapes stream the weights through shared memory
+    static const int use_stream = env_int("PD_GEMV_STREAM", 1);
+    if (use_stream && ws != nullptr && group_offsets == nullptr && d_in % 128 == 0 && ldx % 64 == 0)
+        return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, stream);
     GemvArgs args;
     args.x = x;
     args.w_b = w_b;
