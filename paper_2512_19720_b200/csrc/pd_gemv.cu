@@ -238,61 +238,78 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming decode kernel: weights brought in by TMA, one CTA per 32 output rows, two CTAs per SM.
+// Streaming decode kernel: weights brought in by TMA, one CTA per 16 output rows, two CTAs per SM.
 //
-// A CTA owns 32 rows for the whole of d_in, so its result needs no other CTA: no partial sums in
-// global memory, no tickets, no fences.  It walks d_in in steps of 256 columns; a step is 16 KB of
-// W_b (one TMA box of four 64-column blocks, 128-byte swizzle), 1 KB of mask, the matching 256
-// columns of x and, for the col axis, of v: four TMA instructions per step.  One producer lane keeps
-// a ring of four steps in flight (64 KB of weights per CTA, 128 KB per SM), so an SM's whole share of
-// a 7B-sized layer is requested within the first microsecond.  Fewer CTAs than SMs (4096 rows = 128
-// CTAs) is fine: HBM, not the SM count, is the limit, and an SM with deep queues can pull well above
-// its fair share.
+// A CTA owns 16 rows for the whole of d_in, so its result needs no other CTA: no partial sums in
+// global memory, no tickets, no fences.  It walks d_in in steps of 1024 columns: 2 KB of contiguous
+// W_b per row and step (long row segments are what HBM delivers fastest: on B200 a pure TMA stream
+// of [16 rows x 2 KB] steps, three in flight per CTA, measured 6.1-7.1 TB/s on the 7B shapes,
+// against 4.4-5.4 TB/s for 512-byte segments).  A step is four TMA boxes of {64 columns, 4 blocks,
+// 16 rows} (128-byte swizzle; rows of 512 bytes keep the fragment reads conflict free) plus one box
+// of mask words: 34 KB, three steps in flight per CTA.
 //
-// Eight consumer warps: warp pair p takes the steps s = p (mod 4), which always sit in stage p, so a
-// warp sees every phase of the barriers it waits on in order; inside a pair each warp takes two of
-// the four column blocks and all 32 rows (four n8 tiles), so an x fragment read from shared memory
-// feeds four tiles.  16-byte pieces are read conflict free from the swizzled tiles: lane (g,t)
-// takes pieces t and t+4 of row g of a block.  The eight partial accumulators are added in warp order
-// through shared memory (the buffer reuses the drained ring).
+// Eight consumer warps share every step: warp w takes the 64-column blocks 2w and 2w+1 and both n8
+// tiles.  W_b and mask come from shared memory; the x fragments (and v for the col axis) are read
+// straight from global memory -- x is small and L2-resident, and keeping it out of shared memory
+// leaves the ring to the weights.  The delta term enters the same accumulator as x . (+-s) with
+// s = v[row] (row axis; exact fp16 products summed in fp32) or as (x*v) . (+-1) (col axis).
+// The eight warps' partial sums are added in warp order through shared memory.
 //
-// Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the
-// stream, so their loads are issued before griddepcontrol.wait; x is loaded and y stored after it.
-constexpr int kStreamRows = 32;
-constexpr int kStreamK = 256;
-constexpr int kStreamStages = 4;
+// Programmatic dependent launch: W_b and mask do not depend on the previous kernel in the stream,
+// so the producer starts loading at once; the consumers wait for the previous kernel
+// (griddepcontrol.wait) before they touch x, v or y.
+constexpr int kStreamRows = 16;
+constexpr int kStreamK = 1024;
+constexpr int kStreamStages = 3;
 constexpr int kStreamConsumers = 8;
 constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
-constexpr int kStW = 0;                     // [32 rows][4 blocks][128 B], swizzled
-constexpr int kStX = 16384;                 // [16 rows][4 blocks][128 B], swizzled
-constexpr int kStMask = kStX + 8192;        // [32 rows][8 words]
-constexpr int kStV = kStMask + 1024;        // 256 fp16 (col axis)
-constexpr int kStageBytes = 26 * 1024;      // rounded up: every stage starts 1024-byte aligned
-constexpr int kRedOffset = 0;               // [8 warps][16 tokens][32 rows] fp32, over the ring once it has drained
-constexpr int kBarOffset = kStreamStages * kStageBytes;
+constexpr int kStW = 0;                     // 4 boxes of [16 rows][4 blocks][128 B], swizzled (8 KB each)
+constexpr int kStMask = 32768;              // [16 rows][32 words]
+constexpr int kStageBytes = 34 * 1024;      // every stage starts 1024-byte aligned
+constexpr int kRedOffset = kStreamStages * kStageBytes;  // [8 warps][16 tokens][16 rows] fp32
+constexpr int kBarOffset = kRedOffset + kStreamConsumers * 16 * kStreamRows * 4;
 constexpr int kStreamSmem = kBarOffset + 256 + 1024 /* alignment slack */;
-static_assert(kStreamStages == 4, "stage p belongs to warp pair p");
-static_assert(kStreamConsumers * 16 * kStreamRows * 4 <= kStreamStages * kStageBytes, "reduction buffer must fit the ring");
 
 struct StreamArgs {
+    const __half *x;
     const __half *v;
     __half *y;
-    int64_t ldy;
+    int64_t ldx, ldy;
     int M, d_out, d_in;
-    int n_k;  // steps of 256 columns (the last one may be half empty)
+    int n_k;      // steps of 1024 columns (the last one may be partly past d_in)
     uint32_t *status;
 };
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+
+__device__ __forceinline__ uint4 ldg_cached(const void *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// x fragments of one 64-column block: [c] = piece t + 4c; a = token g, b = token g + 8, v = scales (col axis)
+struct XFrag {
+    uint4 a[2], b[2], v[2];
+};
+
+template <bool COL, bool M16>
+__device__ __forceinline__ void load_xfrag(XFrag &f, const StreamArgs &a, int k0, int g, int t) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const int k = k0 + 8 * (t + 4 * c);
+        f.a[c] = make_uint4(0, 0, 0, 0);
+        f.b[c] = make_uint4(0, 0, 0, 0);
+        if (g < a.M) f.a[c] = ldg_cached(a.x + static_cast<size_t>(g) * a.ldx + k);
+        if (M16 && g + 8 < a.M) f.b[c] = ldg_cached(a.x + static_cast<size_t>(g + 8) * a.ldx + k);
+        if (COL) f.v[c] = ldg_cached(a.v + k);
+    }
 }
 
 template <int AXIS, bool HAS_DELTA, bool M16>
-__global__ void __maxnreg__(112)
-gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                   const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
+__global__ void __maxnreg__(96)
+gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float *red = reinterpret_cast<float *>(smem + kRedOffset);
@@ -301,15 +318,13 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + kStreamStages);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row0 = blockIdx.x * kStreamRows;
     constexpr bool kCol = HAS_DELTA && AXIS == PD_AXIS_COL;
-    constexpr uint32_t kWBytes = 16384u + (HAS_DELTA ? 1024u : 0u);
-    constexpr uint32_t kXBytes = M16 ? 8192u : 4096u;
+    constexpr uint32_t kTxBytes = 32768u + (HAS_DELTA ? 2048u : 0u);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) {
             mbar_init(full + s, 1);
-            mbar_init(empty + s, 2);
+            mbar_init(empty + s, kStreamConsumers);
         }
         *abort_flag = 0;
         mbar_fence_init();
@@ -320,133 +335,140 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // ------------------------------------------------ producer
         if (lane == 0) {
             grid_launch_dependents();  // the next kernel in the stream may start its own weight loads
-            // bytes of v in step s (the last step of a d_in that is not a multiple of 256 has 128 columns)
-            auto v_bytes = [&](int s) { return static_cast<uint32_t>(min(kStreamK, a.d_in - s * kStreamK) * 2); };
-            auto load_w = [&](int s, int st) {
-                unsigned char *base = smem + st * kStageBytes;
-                tma_load_3d(&map_w, full + st, base + kStW, 0, s * 4, row0);
-                if (HAS_DELTA) tma_load_2d(&map_m, full + st, base + kStMask, s * 8, row0);
-                if (kCol) bulk_load_1d(base + kStV, a.v + static_cast<size_t>(s) * kStreamK, v_bytes(s), full + st);
-            };
-            auto load_x = [&](int s, int st) { tma_load_3d(&map_x, full + st, smem + st * kStageBytes + kStX, 0, s * 4, 0); };
-            const int pre = min(a.n_k, kStreamStages);
-            for (int s = 0; s < pre; ++s) {  // weights first: they do not depend on earlier work in the stream
-                mbar_expect_tx(full + s, kWBytes + (kCol ? v_bytes(s) : 0u));
-                load_w(s, s);
-            }
-            grid_dependency_wait();  // x may be the previous kernel's output
-            for (int s = 0; s < pre; ++s) {
-                mbar_arrive_expect_tx(full + s, kXBytes);
-                load_x(s, s);
-            }
-            for (int s = pre; s < a.n_k; ++s) {
-                const int st = s % kStreamStages;
-                if (!mbar_wait(empty + st, ((s / kStreamStages) & 1) ^ 1, abort_flag, a.status, 11)) break;
-                mbar_arrive_expect_tx(full + st, kWBytes + kXBytes + (kCol ? v_bytes(s) : 0u));
-                load_w(s, st);
-                load_x(s, st);
+            uint32_t gs = 0;           // steps issued so far
+            bool ok = true;
+            {
+                const int row0 = blockIdx.x * kStreamRows;
+                for (int s = 0; s < a.n_k; ++s, ++gs) {
+                    const int st = gs % kStreamStages;
+                    if (gs >= kStreamStages &&
+                        !(ok = mbar_wait(empty + st, ((gs / kStreamStages) & 1) ^ 1, abort_flag, a.status, 11)))
+                        break;
+                    unsigned char *base = smem + st * kStageBytes;
+                    mbar_arrive_expect_tx(full + st, kTxBytes);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tma_load_3d(&map_w, full + st, base + kStW + q * 8192, 0, s * 16 + 4 * q, row0);
+                    if (HAS_DELTA) tma_load_2d(&map_m, full + st, base + kStMask, s * 32, row0);
+                }
             }
         }
     } else {
         // ------------------------------------------------ consumers
         const int g = lane >> 2, t = lane & 3;
-        const int pair = warp >> 1, half = warp & 1;  // stage / steps of this pair; which two column blocks
         const uint32_t sel_t = static_cast<uint32_t>(t | ((4 + t) << 4));
-        // One accumulator per tile: the delta term enters as x . (+-s) with s = v[row] (row axis, exact
-        // fp16 products summed in fp32) or as (x*v) . (+-1) (col axis).
-        float acc[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
-        uint32_t mag[4];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            mag[j] = 0x3C003C00u;
-            if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
-                const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
-                mag[j] = h | (h << 16);
-            }
-        }
+        grid_dependency_wait();  // x may be the previous kernel's output
+        const int n_items = 2 * a.n_k;
+        auto item_k0 = [&](int it) { return (it >> 1) * kStreamK + (2 * warp + (it & 1)) * 64; };
+        uint32_t gs = 0;  // steps consumed so far
         bool ok = true;
-        const unsigned char *base = smem + pair * kStageBytes;
-        for (int s = pair; s < a.n_k; s += 4) {
-            if (!(ok = mbar_wait(full + pair, (s / kStreamStages) & 1, abort_flag, a.status, 12))) break;
-            uint32_t my[4];  // per tile: byte 2*b + c = sign bits of piece t + 4c of this warp's block b
-            if (HAS_DELTA) {
+        do {  // one tile per CTA
+            const int row0 = blockIdx.x * kStreamRows;
+            float acc[2][4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 m = *reinterpret_cast<const uint4 *>(base + kStMask + (8 * j + g) * 32 + half * 16);
-                    my[j] = prmt(prmt(m.x, m.y, sel_t), prmt(m.z, m.w, sel_t), 0x5410u);
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
+            uint32_t mag[2];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                mag[j] = 0x3C003C00u;
+                if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
+                    const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
+                    mag[j] = h | (h << 16);
                 }
             }
+            // items: (step s, block bb of this warp), k0 = s*1024 + (2*warp + bb)*64; x fragments one item ahead
+            XFrag cur, nxt;
+            if (item_k0(0) < a.d_in) load_xfrag<kCol, M16>(cur, a, item_k0(0), g, t);
+            for (int it = 0; it < n_items && ok; ++it) {
+                const int bb = it & 1, st = gs % kStreamStages;
+                const int k0 = item_k0(it);
+                if (it + 1 < n_items && item_k0(it + 1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(it + 1), g, t);
+                if (bb == 0 && !(ok = mbar_wait(full + st, (gs / kStreamStages) & 1, abort_flag, a.status, 12))) break;
+                if (k0 < a.d_in) {  // else past the end of d_in: W was zero-filled there and x must not be read
+                    const int blk = 2 * warp + bb;                       // block inside the step
+                    const unsigned char *box = smem + st * kStageBytes + kStW + (blk >> 2) * 8192;
+                    const int bi = blk & 3;                               // block inside its box
+                    uint32_t my[2];                                       // per tile: byte c = sign bits of piece t + 4c
+                    if (HAS_DELTA) {
 #pragma unroll
-            for (int b = 0; b < 2; ++b) {
-                const int blk = 2 * half + b;
-                if (s * kStreamK + blk * 64 >= a.d_in) continue;  // past the end of d_in: nothing was loaded there
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    // byte offset inside a row of the box, swizzled: piece index ^ (bits 7..9 of the offset)
-                    const uint32_t piece = static_cast<uint32_t>(t + 4 * c);
-                    const uint32_t in_row = static_cast<uint32_t>(blk * 128) + ((piece ^ static_cast<uint32_t>(((g & 1) << 2) | blk)) << 4);
-                    const uint4 xa = *reinterpret_cast<const uint4 *>(base + kStX + g * 512 + in_row);
-                    uint4 xb = make_uint4(0, 0, 0, 0);
-                    if (M16) xb = *reinterpret_cast<const uint4 *>(base + kStX + (g + 8) * 512 + in_row);
-                    uint4 da = xa, db = xb;
-                    if (kCol) {
-                        const uint4 vv = *reinterpret_cast<const uint4 *>(base + kStV + blk * 128 + (piece << 4));
-                        da = make_uint4(hmul2_u32(xa.x, vv.x), hmul2_u32(xa.y, vv.y), hmul2_u32(xa.z, vv.z), hmul2_u32(xa.w, vv.w));
-                        if (M16) db = make_uint4(hmul2_u32(xb.x, vv.x), hmul2_u32(xb.y, vv.y), hmul2_u32(xb.z, vv.z), hmul2_u32(xb.w, vv.w));
+                        for (int j = 0; j < 2; ++j) {
+                            const uint2 m = *reinterpret_cast<const uint2 *>(smem + st * kStageBytes + kStMask + (8 * j + g) * 128 + blk * 8);
+                            my[j] = prmt(m.x, m.y, sel_t);
+                        }
                     }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint4 w = *reinterpret_cast<const uint4 *>(base + kStW + (8 * j + g) * 512 + in_row);
-                        mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                        mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
-                        if (HAS_DELTA) {
-                            // pair r = halves 2r, 2r+1 of the piece: bit 2r of byte i -> bit 15, bit 2r+1 -> bit 31;
-                            // a clear bit (B = -1) flips the sign of the magnitude
-                            const int i = 2 * b + c;
-                            const uint32_t sel = static_cast<uint32_t>(((i | 8) << 4) | (((4 + i) | 8) << 12));
-                            uint32_t pm[4];
+                    for (int c = 0; c < 2; ++c) {
+                        // byte offset inside a 512-byte row of the box, swizzled: piece index ^ (bits 7..9 of the offset)
+                        const uint32_t in_row = static_cast<uint32_t>(bi * 128) +
+                                                ((static_cast<uint32_t>(t + 4 * c) ^ static_cast<uint32_t>(((g & 1) << 2) | bi)) << 4);
+                        const uint4 xa = cur.a[c], xb = cur.b[c];
+                        uint4 da = xa, db = xb;
+                        if (kCol) {
+                            const uint4 vv = cur.v[c];
+                            da = make_uint4(hmul2_u32(xa.x, vv.x), hmul2_u32(xa.y, vv.y), hmul2_u32(xa.z, vv.z), hmul2_u32(xa.w, vv.w));
+                            if (M16) db = make_uint4(hmul2_u32(xb.x, vv.x), hmul2_u32(xb.y, vv.y), hmul2_u32(xb.z, vv.z), hmul2_u32(xb.w, vv.w));
+                        }
 #pragma unroll
-                            for (int r = 0; r < 4; ++r)
-                                pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mag[j]);
-                            mma16816(acc[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
-                            mma16816(acc[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
+                        for (int j = 0; j < 2; ++j) {
+                            const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
+                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                            if (HAS_DELTA) {
+                                // pair r = halves 2r, 2r+1 of the piece: bit 2r of byte c -> bit 15, bit 2r+1 -> bit 31;
+                                // a clear bit (B = -1) flips the sign of the magnitude
+                                const uint32_t sel = static_cast<uint32_t>(((c | 8) << 4) | (((4 + c) | 8) << 12));
+                                uint32_t pm[4];
+#pragma unroll
+                                for (int r = 0; r < 4; ++r)
+                                    pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mag[j]);
+                                mma16816(acc[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
+                                mma16816(acc[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
+                            }
                         }
                     }
                 }
+                if (bb == 1) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty + st);
+                    ++gs;
+                }
+                cur = nxt;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty + pair);
-        }
 
-        // ---- add the eight warps' partial sums in warp order (the buffer reuses the ring: every step
-        // has been consumed once all consumer warps are past this barrier)
-        asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
-        if (ok) {
-            float *mine = red + warp * 16 * kStreamRows;
+            // ---- add the eight warps' partial sums in warp order.  The first barrier ORs "a wait ran out"
+            // over the consumers, so that all of them leave together.
+            uint32_t gave_up;
+            asm volatile(
+                "{\n"
+                ".reg .pred p, q;\n"
+                "setp.ne.u32 q, %1, 0;\n"
+                "bar.red.or.pred p, 1, %2, q;\n"
+                "selp.u32 %0, 1, 0, p;\n"
+                "}\n"
+                : "=r"(gave_up)
+                : "r"(static_cast<uint32_t>(!ok || *abort_flag)), "n"(kStreamConsumers * 32)
+                : "memory");
+            if (gave_up) break;
+            float *mine = red + warp * 16 * kStreamRows;  // [16 tokens][16 rows]
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < 2; ++j)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int ol = 8 * j + 2 * t + e;
                     mine[g * kStreamRows + ol] = acc[j][e];
                     mine[(g + 8) * kStreamRows + ol] = acc[j][2 + e];
                 }
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
-        if (!*abort_flag) {
-            grid_dependency_wait();
-            for (int idx = threadIdx.x; idx < 16 * kStreamRows; idx += kStreamConsumers * 32) {
-                const int tok = idx / kStreamRows, ol = idx - tok * kStreamRows;
+            asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
+            {
+                const int idx = threadIdx.x;  // 256 consumer threads = 16 tokens x 16 rows
+                const int tok = idx >> 4, ol = idx & 15;
                 float sum = 0.f;
 #pragma unroll
                 for (int w = 0; w < kStreamConsumers; ++w) sum += red[(w * 16 + tok) * kStreamRows + ol];
                 if (tok < a.M && row0 + ol < a.d_out) a.y[static_cast<size_t>(tok) * a.ldy + row0 + ol] = __float2half_rn(sum);
             }
-        }
+        } while (false);
     }
 }
 
@@ -537,8 +559,8 @@ pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) 
 }
 
 template <int AXIS, bool HAS_DELTA, bool M16>
-pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mx, const CUtensorMap &mm, const StreamArgs &args,
-                                int grid, cudaStream_t stream) {
+pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, const StreamArgs &args, int grid,
+                                cudaStream_t stream) {
     auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16>;
     static bool configured = false;  // per instantiation
     if (!configured) {
@@ -558,32 +580,34 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mx, co
     static const int use_pdl = env_int("PD_PDL", 1);
     cfg.numAttrs = use_pdl ? 1 : 0;
     count_launch();
-    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, mm, args));
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mm, args));
 }
 
 pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                         int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
                         cudaStream_t stream) {
     const bool m16 = M > 8, delta = mask != nullptr;
-    CUtensorMap mw, mx, mm;
-    if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, kStreamRows) ||
-        !make_map_blocked_f16(&mx, x, M, d_in, ldx * 2, 4, m16 ? 16 : 8))
-        return PD_ERR_CUDA;
+    CUtensorMap mw, mm;
+    if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, kStreamRows)) return PD_ERR_CUDA;
     mm = mw;
-    if (delta && !make_map_2d(&mm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, mask, d_out, d_in / 32, d_in / 8, 8, kStreamRows,
+    if (delta && !make_map_2d(&mm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, mask, d_out, d_in / 32, d_in / 8, 32, kStreamRows,
                               CU_TENSOR_MAP_SWIZZLE_NONE))
         return PD_ERR_CUDA;
     StreamArgs a;
+    a.x = x;
     a.v = v;
     a.y = y;
+    a.ldx = ldx;
     a.ldy = ldy;
     a.M = M;
     a.d_out = static_cast<int>(d_out);
     a.d_in = static_cast<int>(d_in);
     a.n_k = static_cast<int>((d_in + kStreamK - 1) / kStreamK);
     a.status = status;
+    // one CTA per tile of 16 rows: a persistent grid walking several tiles measured slower on the 7B
+    // shapes (fewer rings in flight, more registers)
     const int grid = static_cast<int>((d_out + kStreamRows - 1) / kStreamRows);
-#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W>(mw, mx, mm, a, grid, stream)
+#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W>(mw, mm, a, grid, stream)
     if (!delta) {
         if (m16) PD_STREAM_CASE(PD_AXIS_ROW, false, true);
         PD_STREAM_CASE(PD_AXIS_ROW, false, false);
@@ -605,7 +629,7 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       cudaStream_t stream) {
     // plain calls on TMA-friendly shapes stream the weights through shared memory
     static const int use_stream = env_int("PD_GEMV_STREAM", 1);
-    if (use_stream && ws != nullptr && group_offsets == nullptr && d_in % 128 == 0 && ldx % 64 == 0)
+    if (use_stream && ws != nullptr && group_offsets == nullptr && d_in % 128 == 0)
         return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, stream);
     GemvArgs args;
     args.x = x;
