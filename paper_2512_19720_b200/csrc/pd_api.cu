@@ -5,6 +5,8 @@
 #include "pd_common.cuh"
 
 namespace pd {
+size_t grouped_table_bytes(int64_t M, int32_t V);
+
 namespace {
 
 constexpr int kMaxVariants = 64;
@@ -19,7 +21,8 @@ constexpr size_t kOffsetsBytes = 512;
 
 __global__ void __launch_bounds__(kGroupThreads)
 group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict__ offsets,
-                  int *__restrict__ row_index, uint32_t *__restrict__ status) {
+                  int *__restrict__ row_index, uint32_t *__restrict__ status, int4 *__restrict__ tile_table,
+                  int *__restrict__ n_token_tiles) {
     __shared__ int warp_sums[kGroupThreads / 32];
     __shared__ int s_base;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -54,6 +57,25 @@ group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict
         __syncthreads();
         if (threadIdx.x == 0) offsets[grp + 1] = s_base;
     }
+    if (tile_table != nullptr && threadIdx.x == 0) {
+        // cut every bucket into token tiles (thread 0 wrote the offsets itself, so it may read them back)
+        int n = 0;
+        for (int grp = 0; grp <= V; ++grp)
+            for (int first = offsets[grp]; first < offsets[grp + 1]; first += kGroupedTokenTile)
+                tile_table[n++] = make_int4(grp, first, min(kGroupedTokenTile, offsets[grp + 1] - first), 0);
+        *n_token_tiles = n;
+    }
+}
+
+// x_sorted[i, :] = x[row_index[i], :], 16 bytes per thread
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const __half *__restrict__ x, int64_t ldx, int M, int vec_per_row, const int *__restrict__ row_index,
+                   uint4 *__restrict__ x_sorted) {
+    const int64_t total = static_cast<int64_t>(M) * vec_per_row;
+    for (int64_t i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
+        const int r = static_cast<int>(i / vec_per_row), c = static_cast<int>(i - static_cast<int64_t>(r) * vec_per_row);
+        x_sorted[i] = *reinterpret_cast<const uint4 *>(x + static_cast<size_t>(row_index[r]) * ldx + 8 * c);
+    }
 }
 
 pd_status check_matrix_args(const void *x, int64_t M, int64_t ldx, const void *w_b, int64_t d_out, int64_t d_in,
@@ -68,10 +90,24 @@ pd_status check_matrix_args(const void *x, int64_t M, int64_t ldx, const void *w
 }  // namespace
 
 pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,
-                            cudaStream_t stream) {
-    group_rows_kernel<<<1, kGroupThreads, 0, stream>>>(ids, M, V, offsets, row_index, status);
+                            int4 *tile_table, int *n_token_tiles, const __half *x, int64_t ldx, int64_t d_in,
+                            __half *x_sorted, cudaStream_t stream) {
+    group_rows_kernel<<<1, kGroupThreads, 0, stream>>>(ids, M, V, offsets, row_index, status, tile_table, n_token_tiles);
     count_launch();
+    if (x_sorted != nullptr) {
+        const int vec_per_row = static_cast<int>(d_in / 8);
+        const int64_t blocks = (static_cast<int64_t>(M) * vec_per_row + 255) / 256;
+        gather_rows_kernel<<<static_cast<unsigned>(blocks < 4096 ? blocks : 4096), 256, 0, stream>>>(
+            x, ldx, M, vec_per_row, row_index, reinterpret_cast<uint4 *>(x_sorted));
+        count_launch();
+    }
     return cuda_ok(cudaGetLastError());
+}
+
+// workspace of pd_linear_multivariant beyond the status words, offsets and row index (tensor-core path only)
+size_t grouped_table_bytes(int64_t M, int32_t V) {
+    const size_t max_tiles = static_cast<size_t>(M / kGroupedTokenTile + V + 2);
+    return round_up(max_tiles * sizeof(int4), 256) + 256;  // tile table + the tile count
 }
 
 }  // namespace pd
@@ -87,8 +123,9 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
         case PD_OP_LINEAR:
             return kStatusBytes;
         case PD_OP_LINEAR_MULTIVARIANT:
-            (void)V;
-            return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M > 0 ? M : 0), 256);
+            if (M <= 0 || V <= 0) return kStatusBytes + kOffsetsBytes;
+            return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256) +
+                   (M > kGemvMaxTokens ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
         case PD_OP_MERGE:
         default:
             return 0;
@@ -184,11 +221,28 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
     auto *status = reinterpret_cast<uint32_t *>(base);
     int *offsets = reinterpret_cast<int *>(base + kStatusBytes);
     int *row_index = reinterpret_cast<int *>(base + kStatusBytes + kOffsetsBytes);
-    st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, stream);
-    if (st != PD_OK) return st;
     const __half *xh = static_cast<const __half *>(x);
     const __half *vh = static_cast<const __half *>(vs);
     const int64_t mask_words = d_out * (d_in / 32);
+    if (M > kGemvMaxTokens && d_in >= 64) {
+        // prefill-sized batch: sort the rows by variant, gather them, one grouped tensor-core launch
+        unsigned char *p = base + kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256);
+        int4 *tile_table = reinterpret_cast<int4 *>(p);
+        int *n_token_tiles = reinterpret_cast<int *>(p + grouped_table_bytes(M, V) - 256);
+        __half *x_sorted = reinterpret_cast<__half *>(p + grouped_table_bytes(M, V));
+        unsigned long long col_bits = 0;
+        for (int g = 0; g < V; ++g)
+            if (axes[g] == PD_AXIS_COL) col_bits |= 1ull << g;
+        st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, tile_table, n_token_tiles, xh,
+                               ldx, d_in, x_sorted, stream);
+        if (st != PD_OK) return st;
+        return launch_gemm_grouped(x_sorted, M, static_cast<const __half *>(w_b), masks, mask_words, vh, v_stride, col_bits,
+                                   V, d_out, d_in, static_cast<__half *>(y), ldy, tile_table, n_token_tiles,
+                                   static_cast<int>(M / kGroupedTokenTile + V + 2), row_index, status, stream);
+    }
+    st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, nullptr, nullptr, nullptr, 0, 0,
+                           nullptr, stream);
+    if (st != PD_OK) return st;
     for (int g = 0; g <= V; ++g) {
         const bool base_only = (g == V);
         st = launch_gemv(xh, 0, ldx, static_cast<const __half *>(w_b), base_only ? nullptr : masks + g * mask_words,

@@ -40,7 +40,47 @@ struct GemmArgs {
     int M, d_out, d_in;
     int tiles_m, tiles_n, k_steps;
     uint32_t *status;
+    // grouped (multi-variant) mode: the token rows of x are already sorted by variant; token tile i is
+    // tile_table[i] = {variant, first sorted row, rows, 0}; variant V means "base only"
+    const int4 *tile_table;
+    const int *n_token_tiles;   // device: number of entries of tile_table
+    const int *row_index;       // sorted row -> row of y
+    int64_t mask_stride, v_stride;  // elements between two variants' masks / scale vectors
+    unsigned long long col_axis_bits;  // bit g set: variant g scales along d_in
+    int V;
 };
+
+struct Tile {
+    int tm, tok0, count;    // W row tile; first token row (of x); valid tokens
+    const uint32_t *mask;
+    const __half *v;
+    bool col, delta;
+};
+
+template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
+__device__ __forceinline__ Tile get_tile(const GemmArgs &a, int tile, int n_tt) {
+    Tile t;
+    t.tm = tile / n_tt;
+    const int tn = tile - t.tm * n_tt;
+    if (!GROUPED) {
+        t.tok0 = tn * BN;
+        t.count = min(BN, a.M - t.tok0);
+        t.mask = a.mask;
+        t.v = a.v;
+        t.col = AXIS == PD_AXIS_COL;
+        t.delta = HAS_DELTA;
+    } else {
+        const int4 e = __ldg(a.tile_table + tn);
+        t.tok0 = e.y;
+        t.count = e.z;
+        t.delta = e.x < a.V;
+        const int g = t.delta ? e.x : 0;
+        t.mask = a.mask + static_cast<size_t>(g) * a.mask_stride;
+        t.v = a.v + static_cast<size_t>(g) * a.v_stride;
+        t.col = (a.col_axis_bits >> g) & 1ull;
+    }
+    return t;
+}
 
 // ------------------------------------------------------------------ tcgen05 wrappers
 __device__ __forceinline__ void tcgen05_alloc(uint32_t *dst_smem, uint32_t cols) {
@@ -101,7 +141,7 @@ struct SmemLayout {
     static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
 };
 
-template <int AXIS, bool HAS_DELTA, int BN>
+template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = SmemLayout<BN>;
@@ -114,7 +154,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = a.tiles_m * a.tiles_n;
+    const int n_tt = GROUPED ? __ldg(a.n_token_tiles) : a.tiles_n;  // token tiles
+    const int n_tiles = a.tiles_m * n_tt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -141,24 +182,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int tm = tile / a.tiles_n, tn = tile - tm * a.tiles_n;
+                const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                     const int s = it % kStages;
                     if (!(ok = mbar_wait(empty + s, ((it / kStages) & 1) ^ 1, abort_flag, a.status, 1))) break;
                     unsigned char *st = smem + s * L::kStageBytes;
                     mbar_arrive_expect_tx(full + s, L::kStageBytes);
-                    tma_load_2d(&map_w, full + s, st, ks * BK, tm * BM);
-                    tma_load_2d(&map_x, full + s, st + L::kWBytes, ks * BK, tn * BN);
+                    tma_load_2d(&map_w, full + s, st, ks * BK, ti.tm * BM);
+                    tma_load_2d(&map_x, full + s, st + L::kWBytes, ks * BK, ti.tok0);
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+                // MMA N = the tile's tokens rounded up to 16 (the whole 256-token box in the plain mode)
+                const int n_mma = GROUPED ? ((get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt).count + 15) & ~15) : BN;
+                const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
                 const uint32_t b = tcount & 1;
                 if (!(ok = mbar_wait(acc_empty + b, ((tcount >> 1) & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
@@ -186,23 +229,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         uint32_t tcount = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
-            const int tm = tile / a.tiles_n, tn = tile - tm * a.tiles_n;
+            const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
             const uint32_t b = tcount & 1;
             if (!(ok = mbar_wait(acc_full + b, (tcount >> 1) & 1, abort_flag, a.status, 4))) break;
             tcgen05_fence_after();
-            const int o = tm * BM + quarter * 32 + lane;
+            const int o = ti.tm * BM + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * kAccCols;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (c0 >= ti.count) break;  // warp-uniform: no token of this tile lives in these columns
                 uint32_t r[32];
                 tcgen05_ld_32x32b_x32(taddr + c0, r);
                 tcgen05_wait_ld();
-                const int tok0 = tn * BN + c0;
                 if (o < a.d_out) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (tok0 + j < a.M)
-                            a.y[static_cast<size_t>(tok0 + j) * a.ldy + o] = __float2half_rn(__uint_as_float(r[j]));
+                        if (c0 + j < ti.count) {
+                            const int yr = GROUPED ? __ldg(a.row_index + ti.tok0 + c0 + j) : ti.tok0 + c0 + j;
+                            a.y[static_cast<size_t>(yr) * a.ldy + o] = __float2half_rn(__uint_as_float(r[j]));
+                        }
                     }
                 }
             }
@@ -218,26 +263,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int tm = tile / a.tiles_n;
-            const int o = tm * BM + r;
+            const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
+            const bool delta = ti.delta, col = ti.col;  // compile-time constants in the plain mode
+            const int o = ti.tm * BM + r;
             const bool row_ok = o < a.d_out;
             uint32_t vrow = 0;
-            if (HAS_DELTA && AXIS == PD_AXIS_ROW && row_ok) {
-                const uint32_t hv = *reinterpret_cast<const unsigned short *>(a.v + o);
+            if (delta && !col && row_ok) {
+                const uint32_t hv = *reinterpret_cast<const unsigned short *>(ti.v + o);
                 vrow = hv | (hv << 16);
             }
-            const uint32_t *mrow = HAS_DELTA ? a.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
+            const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
             uint32_t word_next = 0;
-            if (HAS_DELTA && row_ok && h < words) word_next = __ldg(mrow + h);
+            if (delta && row_ok && h < words) word_next = __ldg(mrow + h);
             for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                 const int s = it % kStages;
                 const uint32_t word = word_next;
-                if (HAS_DELTA) {
+                if (delta) {
                     const int wi = 2 * (ks + 1) + h;
                     word_next = (row_ok && ks + 1 < a.k_steps && wi < words) ? __ldg(mrow + wi) : 0u;
                 }
                 if (!(ok = mbar_wait(full + s, (it / kStages) & 1, abort_flag, a.status, 5))) break;
-                if (HAS_DELTA) {
+                if (delta) {
                     unsigned char *wt = smem + s * L::kStageBytes + r * 128;
                     uint32_t sh[8];
 #pragma unroll
@@ -248,10 +294,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                         uint4 *p = reinterpret_cast<uint4 *>(wt + ((((4 * h + j) ^ (r & 7))) << 4));
                         uint4 w = *p;
                         uint32_t vv[4] = {vrow, vrow, vrow, vrow};
-                        if (AXIS == PD_AXIS_COL) {
+                        if (col) {
                             const int k = kcol + 8 * j;
                             uint4 t4 = make_uint4(0, 0, 0, 0);
-                            if (k < a.d_in) t4 = __ldg(reinterpret_cast<const uint4 *>(a.v + k));
+                            if (k < a.d_in) t4 = __ldg(reinterpret_cast<const uint4 *>(ti.v + k));
                             vv[0] = t4.x; vv[1] = t4.y; vv[2] = t4.z; vv[3] = t4.w;
                         }
                         const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
@@ -294,9 +340,9 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
                        CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int AXIS, bool HAS_DELTA, int BN>
+template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
 pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
-    auto kernel = gemm_kernel<AXIS, HAS_DELTA, BN>;
+    auto kernel = gemm_kernel<AXIS, HAS_DELTA, GROUPED, BN>;
     constexpr int smem = SmemLayout<BN>::kTotal;
     static bool configured = false;
     if (!configured) {
@@ -316,7 +362,7 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
     constexpr int BN = 256;
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, BN)) return PD_ERR_CUDA;
-    GemmArgs args;
+    GemmArgs args = {};
     args.mask = mask;
     args.v = v;
     args.y = y;
@@ -330,9 +376,41 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
     args.status = status;
     const int tiles = args.tiles_m * args.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    if (mask == nullptr) return launch_one<PD_AXIS_ROW, false, BN>(mw, mx, args, grid, stream);
-    if (axis == PD_AXIS_ROW) return launch_one<PD_AXIS_ROW, true, BN>(mw, mx, args, grid, stream);
-    return launch_one<PD_AXIS_COL, true, BN>(mw, mx, args, grid, stream);
+    if (mask == nullptr) return launch_one<PD_AXIS_ROW, false, false, BN>(mw, mx, args, grid, stream);
+    if (axis == PD_AXIS_ROW) return launch_one<PD_AXIS_ROW, true, false, BN>(mw, mx, args, grid, stream);
+    return launch_one<PD_AXIS_COL, true, false, BN>(mw, mx, args, grid, stream);
+}
+
+pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
+                              int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
+                              int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
+                              const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
+                              cudaStream_t stream) {
+    constexpr int BN = kGroupedTokenTile;
+    CUtensorMap mw, mx;
+    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, BN)) return PD_ERR_CUDA;
+    GemmArgs args = {};
+    args.mask = masks;
+    args.v = vs;
+    args.y = y;
+    args.ldy = ldy;
+    args.M = static_cast<int>(M);
+    args.d_out = static_cast<int>(d_out);
+    args.d_in = static_cast<int>(d_in);
+    args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
+    args.tiles_n = 0;
+    args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
+    args.status = status;
+    args.tile_table = tile_table;
+    args.n_token_tiles = n_token_tiles;
+    args.row_index = row_index;
+    args.mask_stride = mask_stride;
+    args.v_stride = v_stride;
+    args.col_axis_bits = col_axis_bits;
+    args.V = V;
+    const int64_t tiles = static_cast<int64_t>(args.tiles_m) * max_token_tiles;  // upper bound; the kernel reads the real count
+    const int grid = tiles < sm_count() ? static_cast<int>(tiles) : sm_count();
+    return launch_one<PD_AXIS_ROW, true, true, BN>(mw, mx, args, grid, stream);
 }
 
 }  // namespace pd

@@ -335,6 +335,29 @@ def test_multivariant_small(api, d_out, d_in, n_var, m):
         assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
 
 
+@pytest.mark.parametrize("d_out,d_in,n_var,m", [(256, 512, 5, 300), (200, 1152, 3, 150), (1024, 1024, 16, 2112), (130, 96, 2, 700)])
+def test_multivariant_prefill_sized(api, d_out, d_in, n_var, m):
+    # more than 64 rows: rows are bucketed by variant and run through the grouped tensor-core kernel
+    w_b = synth.gen_base(d_out, d_in, 21)
+    masks, vs, axes = make_variants(w_b, n_var, 21)
+    x = synth.gen_x(m, d_in, 22)
+    ids = synth.gen_ids(m, n_var, 23)
+    ids[::37] = -1
+    ref, bad = orc.linear_multivariant(x, ids, w_b, masks, vs, axes)
+    assert bad == 0
+    args = (dev(x), dev(ids), dev(w_b), dev(masks), dev(vs), axes)
+    y = api.pd_linear_multivariant(*args)
+    y2 = api.pd_linear_multivariant(*args)
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == 0
+    yh = host(y).astype(np.float64)
+    assert np.isfinite(yh).all()
+    assert rel_err(host(y), ref) <= TOL
+    assert torch.equal(y, y2)
+    for r in range(0, m, 7):  # no row may borrow another variant's delta
+        assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
+
+
 def test_multivariant_bad_id_is_latched(api):
     w_b = synth.gen_base(128, 128, 14)
     masks, vs, axes = make_variants(w_b, 2, 14)
