@@ -26,7 +26,10 @@ namespace {
 constexpr int BM = 128;          // output rows per tile (MMA M)
 constexpr int BK = 64;           // k per stage: 128 bytes of fp16 = one swizzle atom
 constexpr int kStages = 4;
-constexpr int kAccCols = 256;    // TMEM columns per accumulator buffer
+constexpr int kAccCols = 256;    // TMEM columns of the accumulator (one buffer)
+constexpr int kAccBufs = 1;
+constexpr int kACol0 = kAccBufs * kAccCols;  // first TMEM column of the W_hat ring: kStages slots of 32 columns
+constexpr int kVSlotBytes = 128;             // col axis: the 64 scales of a k step
 constexpr int kNumWarps = 14;    // 0 producer, 1 MMA, 2-5 epilogue, 6-13 transform
 constexpr int kNumThreads = kNumWarps * 32;
 constexpr int kXformWarps = 8;
@@ -119,6 +122,28 @@ __device__ __forceinline__ void tcgen05_ld_32x32b_x32(uint32_t taddr, uint32_t (
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tcgen05_mma_f16_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_st_32x32b_x32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
 // 1024 bytes apart; `addr` is the byte address of the first row (plus the k offset inside the atom).
@@ -138,7 +163,8 @@ struct SmemLayout {
     static constexpr int kXBytes = BN * BK * 2;   // 32 KB for BN = 256
     static constexpr int kStageBytes = kWBytes + kXBytes;
     static constexpr int kBarOffset = kStages * kStageBytes;
-    static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+    static constexpr int kVOffset = kBarOffset + 256;        // kStages slots of kVSlotBytes
+    static constexpr int kTotal = kVOffset + kStages * kVSlotBytes + 1024;  // + slack for 1024-byte alignment
 };
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
@@ -160,15 +186,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full + s, 1);
-            mbar_init(xform + s, kXformWarps);
+            mbar_init(xform + s, kXformWarps / 2);  // the four warps (one per TMEM lane quarter) that own the stage
             mbar_init(empty + s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(acc_full + b, 1);
             mbar_init(acc_empty + b, kEpiWarps);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < kStages * kVSlotBytes / 4) {  // scale slots start at zero: a short last k step leaves its tail untouched
+        reinterpret_cast<uint32_t *>(smem + L::kVOffset)[threadIdx.x] = 0u;
+        fence_proxy_async_smem();
     }
     if (warp == 1) tcgen05_alloc(tmem_slot, 512);
     tcgen05_fence_before();
@@ -187,9 +217,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                     const int s = it % kStages;
                     if (!(ok = mbar_wait(empty + s, ((it / kStages) & 1) ^ 1, abort_flag, a.status, 1))) break;
                     unsigned char *st = smem + s * L::kStageBytes;
-                    mbar_arrive_expect_tx(full + s, L::kStageBytes);
+                    const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
+                    mbar_arrive_expect_tx(full + s, L::kStageBytes + v_bytes);
                     tma_load_2d(&map_w, full + s, st, ks * BK, ti.tm * BM);
                     tma_load_2d(&map_x, full + s, st + L::kWBytes, ks * BK, ti.tok0);
+                    if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, full + s);
                 }
             }
         }
@@ -200,10 +232,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
                 // MMA N = the tile's tokens rounded up to 16 (the whole 256-token box in the plain mode)
-                const int n_mma = GROUPED ? ((get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt).count + 15) & ~15) : BN;
+                const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
+                const int n_mma = GROUPED ? ((ti.count + 15) & ~15) : BN;
                 const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
-                const uint32_t b = tcount & 1;
-                if (!(ok = mbar_wait(acc_empty + b, ((tcount >> 1) & 1) ^ 1, abort_flag, a.status, 2))) break;
+                const uint32_t b = tcount % kAccBufs;
+                if (!(ok = mbar_wait(acc_empty + b, ((tcount / kAccBufs) & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + b * kAccCols;
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
@@ -214,9 +247,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                     const uint32_t x_addr = w_addr + L::kWBytes;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk) {
-                        const uint64_t da = make_smem_desc(w_addr + kk * 32);
                         const uint64_t db = make_smem_desc(x_addr + kk * 32);
-                        tcgen05_mma_f16(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                        if (ti.delta)  // A = the W_hat slot the transform warps filled in tensor memory
+                            tcgen05_mma_f16_tmem_a(d_tmem, tmem_base + kACol0 + s * 32 + kk * 8, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                        else           // base only: A = the W_b tile as TMA delivered it
+                            tcgen05_mma_f16(d_tmem, make_smem_desc(w_addr + kk * 32), db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
                     }
                     tcgen05_commit(empty + s);  // frees the stage when these MMAs have read it
                 }
@@ -230,8 +265,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
             const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
-            const uint32_t b = tcount & 1;
-            if (!(ok = mbar_wait(acc_full + b, (tcount >> 1) & 1, abort_flag, a.status, 4))) break;
+            const uint32_t b = tcount % kAccBufs;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(acc_full + b, (tcount / kAccBufs) & 1, abort_flag, a.status, 4)))) break;
             tcgen05_fence_after();
             const int o = ti.tm * BM + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * kAccCols;
@@ -256,10 +291,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             if (lane == 0) mbar_arrive(acc_empty + b);
         }
     } else {
-        // ------------------------------------------------ transform: W_b tile -> W_hat tile, in place
-        const int tt = threadIdx.x - (2 + kEpiWarps) * 32;  // 0..255
-        const int r = tt >> 1, h = tt & 1;                   // tile row, 32-column half of the stage
+        // ------------------------------------------------ transform: W_b tile (shared memory) -> W_hat slot (tensor memory)
+        // A thread owns one row of the tile (its TMEM lane) and all 64 k of a stage; the four warps with
+        // (warp - 6) / 4 == 0 take the even stages, the other four the odd ones.
+        const int quarter = warp & 3;                 // the 32 TMEM lanes this warp may write
+        const uint32_t par = static_cast<uint32_t>((warp - (2 + kEpiWarps)) >> 2);
+        const int r = quarter * 32 + lane;            // tile row
         const int words = a.d_in >> 5;
+        const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -273,48 +312,51 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 vrow = hv | (hv << 16);
             }
             const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
-            uint32_t word_next = 0;
-            if (delta && row_ok && h < words) word_next = __ldg(mrow + h);
-            for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
-                const int s = it % kStages;
-                const uint32_t word = word_next;
+            auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
+                w0 = (delta && row_ok && ks < a.k_steps && 2 * ks < words) ? __ldg(mrow + 2 * ks) : 0u;
+                w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
+            };
+            int ks = static_cast<int>((par ^ it) & 1u);  // first k step of this tile that falls to this warp
+            uint32_t wn0, wn1;
+            load_words(ks, wn0, wn1);
+            for (; ks < a.k_steps; ks += 2) {
+                const uint32_t my_it = it + ks;
+                const int s = my_it % kStages;
+                const uint32_t word[2] = {wn0, wn1};
+                load_words(ks + 2, wn0, wn1);
+                // the TMEM store below is warp-collective: all lanes leave together or not at all
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(full + s, (my_it / kStages) & 1, abort_flag, a.status, 5)))) break;
                 if (delta) {
-                    const int wi = 2 * (ks + 1) + h;
-                    word_next = (row_ok && ks + 1 < a.k_steps && wi < words) ? __ldg(mrow + wi) : 0u;
-                }
-                if (!(ok = mbar_wait(full + s, (it / kStages) & 1, abort_flag, a.status, 5))) break;
-                if (delta) {
-                    unsigned char *wt = smem + s * L::kStageBytes + r * 128;
-                    uint32_t sh[8];
+                    const unsigned char *wt = smem + s * L::kStageBytes + r * 128;
+                    const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
+                    uint32_t out[32];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) sh[q] = word << q;  // bit 8j+q' on top of byte j in sh[7-q']
-                    const int kcol = ks * BK + 32 * h;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 *p = reinterpret_cast<uint4 *>(wt + ((((4 * h + j) ^ (r & 7))) << 4));
-                        uint4 w = *p;
+                    for (int c = 0; c < 8; ++c) {  // 16-byte piece c = columns 8c .. 8c+7 of the stage
+                        const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
                         uint32_t vv[4] = {vrow, vrow, vrow, vrow};
                         if (col) {
-                            const int k = kcol + 8 * j;
-                            uint4 t4 = make_uint4(0, 0, 0, 0);
-                            if (k < a.d_in) t4 = __ldg(reinterpret_cast<const uint4 *>(ti.v + k));
-                            vv[0] = t4.x; vv[1] = t4.y; vv[2] = t4.z; vv[3] = t4.w;
+                            const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
+                            vv[0] = t4.x, vv[1] = t4.y, vv[2] = t4.z, vv[3] = t4.w;
                         }
+                        const uint32_t bits = word[c >> 2];
+                        const int j = c & 3;  // byte of the word that belongs to this piece
                         const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
-                        uint32_t *wp = reinterpret_cast<uint32_t *>(&w);
+                        const uint32_t wp[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                         for (int pr = 0; pr < 4; ++pr) {
-                            // halves 2pr (low) and 2pr+1 (high) of this 8-column piece: +v where the bit is 1, -v where 0
-                            const uint32_t rep = prmt(sh[7 - 2 * pr], sh[6 - 2 * pr], sel);
-                            wp[pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
+                            // halves 2pr (low) and 2pr+1 (high) of the piece: +v where the bit is 1, -v where it is 0
+                            const uint32_t rep = prmt(bits << (7 - 2 * pr), bits << (6 - 2 * pr), sel);
+                            out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
                         }
-                        *p = w;
                     }
-                    fence_proxy_async_smem();
+                    tcgen05_st_32x32b_x32(a_taddr + s * 32, out);
+                    tcgen05_wait_st();
+                    tcgen05_fence_before();
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(xform + s);
             }
+            it += a.k_steps;
         }
     }
 
