@@ -51,6 +51,7 @@ struct GemmArgs {
     int64_t mask_stride, v_stride;  // elements between two variants' masks / scale vectors
     unsigned long long col_axis_bits;  // bit g set: variant g scales along d_in
     int V;
+    int y_vec_ok;  // y is 16-byte aligned and ldy a multiple of 8: rows can be written with 16-byte stores
 };
 
 struct Tile {
@@ -164,7 +165,8 @@ struct SmemLayout {
     static constexpr int kStageBytes = kWBytes + kXBytes;
     static constexpr int kBarOffset = kStages * kStageBytes;
     static constexpr int kVOffset = kBarOffset + 256;        // kStages slots of kVSlotBytes
-    static constexpr int kTotal = kVOffset + kStages * kVSlotBytes + 1024;  // + slack for 1024-byte alignment
+    static constexpr int kOutOffset = kVOffset + kStages * kVSlotBytes;   // epilogue staging: [128 tokens][128 rows] fp16
+    static constexpr int kTotal = kOutOffset + 128 * 128 * 2 + 1024;      // + slack for 1024-byte alignment
 };
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
@@ -259,36 +261,70 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             }
         }
     } else if (warp < 2 + kEpiWarps) {
-        // ------------------------------------------------ epilogue: TMEM -> fp16 -> y[token][row]
+        // ------------------------------------------------ epilogue: TMEM -> fp16 -> shared-memory staging -> y[token][row]
+        // The accumulator is drained in two halves of 128 tokens through a 32 KB staging tile laid out
+        // [token][128 rows], so that y is written with 16-byte stores, 256 contiguous bytes per token; the
+        // accumulator is handed back to the MMA warp as soon as its last column has been read.
         const int quarter = warp & 3;  // the 32 TMEM lanes this warp may read
+        const int et = threadIdx.x - 2 * 32;  // 0..127 among the epilogue threads
+        unsigned char *stage_out = smem + L::kOutOffset;
         uint32_t tcount = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
             const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
             const uint32_t b = tcount % kAccBufs;
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait(acc_full + b, (tcount / kAccBufs) & 1, abort_flag, a.status, 4)))) break;
+            const bool got = mbar_wait(acc_full + b, (tcount / kAccBufs) & 1, abort_flag, a.status, 4);
+            uint32_t gave_up;  // OR over the four epilogue warps, so that they leave together
+            asm volatile(
+                "{\n"
+                ".reg .pred p, q;\n"
+                "setp.ne.u32 q, %1, 0;\n"
+                "bar.red.or.pred p, 2, %2, q;\n"
+                "selp.u32 %0, 1, 0, p;\n"
+                "}\n"
+                : "=r"(gave_up)
+                : "r"(static_cast<uint32_t>(!got)), "n"(kEpiWarps * 32)
+                : "memory");
+            if (gave_up) break;
             tcgen05_fence_after();
-            const int o = ti.tm * BM + quarter * 32 + lane;
+            const int row_l = quarter * 32 + lane;          // row of the tile this thread reads from TMEM
+            const int o0 = ti.tm * BM;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + b * kAccCols;
+            const int n_half = (ti.count + 127) / 128;      // 1 or 2
+            for (int hf = 0; hf < n_half; ++hf) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (c0 >= ti.count) break;  // warp-uniform: no token of this tile lives in these columns
-                uint32_t r[32];
-                tcgen05_ld_32x32b_x32(taddr + c0, r);
-                tcgen05_wait_ld();
-                if (o < a.d_out) {
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    if (hf * 128 + c0 >= ti.count) break;  // warp-uniform: no token of this tile lives in these columns
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(taddr + hf * 128 + c0, r);
+                    tcgen05_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (c0 + j < ti.count) {
-                            const int yr = GROUPED ? __ldg(a.row_index + ti.tok0 + c0 + j) : ti.tok0 + c0 + j;
-                            a.y[static_cast<size_t>(yr) * a.ldy + o] = __float2half_rn(__uint_as_float(r[j]));
-                        }
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<__half *>(stage_out + (c0 + j) * 256 + row_l * 2) = __float2half_rn(__uint_as_float(r[j]));
+                }
+                if (hf == n_half - 1) {  // every column of the accumulator has been read
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_empty + b);
+                }
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                const int n_tok = min(128, ti.count - hf * 128);
+                for (int idx = et; idx < n_tok * 16; idx += kEpiWarps * 32) {
+                    const int tok = idx >> 4, ch = idx & 15;
+                    const int yr = GROUPED ? __ldg(a.row_index + ti.tok0 + hf * 128 + tok) : ti.tok0 + hf * 128 + tok;
+                    const int o = o0 + ch * 8;
+                    __half *dst = a.y + static_cast<size_t>(yr) * a.ldy + o;
+                    const uint4 val = *reinterpret_cast<const uint4 *>(stage_out + tok * 256 + ch * 16);
+                    if (a.y_vec_ok && o + 8 <= a.d_out) {
+                        *reinterpret_cast<uint4 *>(dst) = val;
+                    } else {
+                        const __half *hv = reinterpret_cast<const __half *>(&val);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (o + q < a.d_out) dst[q] = hv[q];
                     }
                 }
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
             }
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty + b);
         }
     } else {
         // ------------------------------------------------ transform: W_b tile (shared memory) -> W_hat slot (tensor memory)
@@ -416,6 +452,7 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
     args.tiles_n = static_cast<int>((M + BN - 1) / BN);
     args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
     args.status = status;
+    args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = args.tiles_m * args.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
     if (mask == nullptr) return launch_one<PD_AXIS_ROW, false, false, BN>(mw, mx, args, grid, stream);
@@ -443,6 +480,7 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
     args.tiles_n = 0;
     args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
     args.status = status;
+    args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     args.tile_table = tile_table;
     args.n_token_tiles = n_token_tiles;
     args.row_index = row_index;
