@@ -1,6 +1,7 @@
 // C ABI of the pd library: argument checks, workspace layout, dispatch.  No device memory is
 // allocated here; everything runs on the caller's stream.
 #include <climits>
+#include <cstdlib>
 
 #include "pd_common.cuh"
 
@@ -125,7 +126,7 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
         case PD_OP_LINEAR_MULTIVARIANT:
             if (M <= 0 || V <= 0) return kStatusBytes + kOffsetsBytes;
             return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256) +
-                   (M > kGemvMaxTokens ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
+                   (M > 16 ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
         case PD_OP_MERGE:
         default:
             return 0;
@@ -224,8 +225,9 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
     const __half *xh = static_cast<const __half *>(x);
     const __half *vh = static_cast<const __half *>(vs);
     const int64_t mask_words = d_out * (d_in / 32);
-    if (M > kGemvMaxTokens && d_in >= 64) {
-        // prefill-sized batch: sort the rows by variant, gather them, one grouped tensor-core launch
+    static const int grouped_min = [] { const char *e = getenv("PD_GROUPED_MIN_M"); return e ? atoi(e) : 17; }();
+    if (M >= grouped_min && d_in >= 64) {
+        // more than one decode chunk: sort the rows by variant, gather them, one grouped tensor-core launch
         unsigned char *p = base + kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256);
         int4 *tile_table = reinterpret_cast<int4 *>(p);
         int *n_token_tiles = reinterpret_cast<int *>(p + grouped_table_bytes(M, V) - 256);

@@ -434,10 +434,12 @@ pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArg
 
 }  // namespace
 
-pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
-                      const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      uint32_t *status, cudaStream_t stream) {
-    constexpr int BN = 256;
+namespace {
+
+template <int BN>
+pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
+                         int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                         cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, BN)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -458,6 +460,29 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
     if (mask == nullptr) return launch_one<PD_AXIS_ROW, false, false, BN>(mw, mx, args, grid, stream);
     if (axis == PD_AXIS_ROW) return launch_one<PD_AXIS_ROW, true, false, BN>(mw, mx, args, grid, stream);
     return launch_one<PD_AXIS_COL, true, false, BN>(mw, mx, args, grid, stream);
+}
+
+}  // namespace
+
+pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
+                      const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
+                      uint32_t *status, cudaStream_t stream) {
+    // 256 tokens per tile amortise the W_hat transform best, but with few tokens that leaves most SMs without
+    // a tile (M = 256 on a 4096-row layer: 32 tiles).  Estimated time = waves x per-stage time, where a stage
+    // costs the MMA (2 clocks per token) but never less than the transform/handshake floor; ties go to the
+    // smaller tile, which spreads the weight stream over more SMs.
+    const int64_t tiles_m = (d_out + BM - 1) / BM;
+    const int sms = sm_count();
+    int best = 256;
+    int64_t best_cost = -1;
+    for (int bn = 256; bn >= 64; bn >>= 1) {
+        const int64_t tiles = tiles_m * ((M + bn - 1) / bn);
+        const int64_t cost = ((tiles + sms - 1) / sms) * (2 * bn > 400 ? 2 * bn : 400);
+        if (best_cost < 0 || cost <= best_cost) best = bn, best_cost = cost;
+    }
+    if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
 }
 
 pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
