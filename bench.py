@@ -193,7 +193,7 @@ def run_ours(args):
     axes = [ROW] * N_VARIANTS
     torch.cuda.synchronize()
 
-    sections = ["pack", "decode", "prefill", "multi", "merge"]
+    sections = ["pack", "decode", "prefill", "multi_decode", "multi_prefill", "merge"]
 
     def run_pack():
         for L in layers:
@@ -205,8 +205,8 @@ def run_ours(args):
                 for L in layers:
                     api.pd_linear(x_all[L["d_in"]][:m], L["w_b"], L["mask"], L["v"][axis], axis, y=y_all[L["d_out"]][:m])
 
-    def run_multi():
-        for m in MULTI_M:
+    def run_multi(m):
+        if True:
             for L in layers:
                 api.pd_linear_multivariant(x_all[L["d_in"]][:m], ids[m], L["w_b"], L["masks"], L["vs"], axes,
                                            y=y_all[L["d_out"]][:m])
@@ -217,7 +217,8 @@ def run_ours(args):
                 api.pd_merge(L["w_b"], L["mask"], L["v"][axis], axis, w_hat=L["w_hat"])
 
     bodies = {"pack": run_pack, "decode": lambda: run_linear(DECODE_M), "prefill": lambda: run_linear(PREFILL_M),
-              "multi": run_multi, "merge": run_merge}
+              "multi_decode": lambda: run_multi(MULTI_M[0]), "multi_prefill": lambda: run_multi(MULTI_M[1]),
+              "merge": run_merge}
 
     # Every section is captured once into a CUDA graph (the calls only enqueue kernels on the current
     # stream) and replayed: a decode kernel lasts ~10 us, less than the host needs to issue it.
@@ -248,10 +249,11 @@ def run_ours(args):
         "pack": sum(pack_bytes(L["d_out"], L["d_in"]) for L in layers),
         "decode": sum(linear_bytes(m, L["d_out"], L["d_in"], ax) for m in DECODE_M for ax in (ROW, COL) for L in layers),
         "prefill": sum(2 * m * L["d_out"] * L["d_in"] for m in PREFILL_M for _ in (ROW, COL) for L in layers),
-        "multi": sum(multi_bytes(m, L["d_out"], L["d_in"]) for m in MULTI_M for L in layers),
+        "multi_decode": sum(multi_bytes(MULTI_M[0], L["d_out"], L["d_in"]) for L in layers),
+        "multi_prefill": sum(2 * MULTI_M[1] * L["d_out"] * L["d_in"] for L in layers),
         "merge": sum(merge_bytes(L["d_out"], L["d_in"], ax) for ax in (ROW, COL) for L in layers),
     }
-    calls_per = {"pack": 7, "decode": 42, "prefill": 42, "multi": 14, "merge": 14}
+    calls_per = {"pack": 7, "decode": 42, "prefill": 42, "multi_decode": 7, "multi_prefill": 7, "merge": 14}
 
     def barrier():
         torch.cuda.synchronize()
@@ -268,7 +270,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(sections) + 1)] for _ in range(args.steps)]
     barrier()
     for k in range(args.steps):
         step(events[k])
@@ -280,7 +282,7 @@ def run_ours(args):
 
     sec_ms = {s: sum(events[k][i].elapsed_time(events[k][i + 1]) for k in range(args.steps)) / args.steps
               for i, s in enumerate(sections)}
-    total_ms = events[0][0].elapsed_time(events[-1][5]) / args.steps
+    total_ms = events[0][0].elapsed_time(events[-1][len(sections)]) / args.steps
 
     # ---- end to end for the headline metric: host x -> device, pd_linear, y -> host, every call
     host_x = {d_in: x_all[d_in][:16].cpu().pin_memory() for d_in in x_all}
@@ -317,8 +319,9 @@ def run_ours(args):
 
     if rank == 0:
         pk = peaks()
-        gbs = {s: work[s] * world / (sec_ms[s] * 1e-3) / 1e9 for s in ("pack", "decode", "multi", "merge")}
+        gbs = {s: work[s] * world / (sec_ms[s] * 1e-3) / 1e9 for s in ("pack", "decode", "multi_decode", "merge")}
         tfl = work["prefill"] * world / (sec_ms["prefill"] * 1e-3) / 1e12
+        tfl_mv = work["multi_prefill"] * world / (sec_ms["multi_prefill"] * 1e-3) / 1e12
 
         def hbm(section, kernel):
             per_gpu = gbs[section] / world
@@ -328,17 +331,21 @@ def run_ours(args):
                     "algorithmic_bytes_per_call": work[section] // calls_per[section],
                     "avg_call_ms": round(sec_ms[section] / calls_per[section], 5),
                     "share_of_step": round(sec_ms[section] / sum(sec_ms.values()), 4)}
-        gemm_roof = {"kernel": "gemm_kernel (tcgen05 prefill)", "bound": "tensor", "achieved": round(tfl / world, 1),
-                     "peak": pk["tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": round(tfl / world / pk["tflops_sustained"], 4), "frac_of": pk["source"] + " sustained",
-                     "frac_of_burst": round(tfl / world / pk["tflops_burst"], 4),
-                     "frac_of_nominal_2250": round(tfl / world / 2250.0, 4), "traffic": None,
-                     "algorithmic_flops_per_call": work["prefill"] // calls_per["prefill"],
-                     "avg_call_ms": round(sec_ms["prefill"] / calls_per["prefill"], 5),
-                     "share_of_step": round(sec_ms["prefill"] / sum(sec_ms.values()), 4)}
+        def tensor(section, tf_total, kernel):
+            per_gpu = tf_total / world
+            return {"kernel": kernel, "bound": "tensor", "achieved": round(per_gpu, 1), "peak": pk["tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": round(per_gpu / pk["tflops_sustained"], 4),
+                    "frac_of": pk["source"] + " sustained (fp16 and bf16 share one tensor peak)",
+                    "frac_of_burst": round(per_gpu / pk["tflops_burst"], 4),
+                    "frac_of_nominal_2250": round(per_gpu / 2250.0, 4), "traffic": None,
+                    "algorithmic_flops_per_call": work[section] // calls_per[section],
+                    "avg_call_ms": round(sec_ms[section] / calls_per[section], 5),
+                    "share_of_step": round(sec_ms[section] / sum(sec_ms.values()), 4)}
+        gemm_roof = tensor("prefill", tfl, "gemm_kernel (tcgen05 prefill)")
         cpu = oracle_sample(4, 1) if (world == 1 and not args.no_cpu_baseline) else None
         all_roofs = {"decode": hbm("decode", "gemv_stream_kernel (decode)"), "pack": hbm("pack", "pack_kernel"),
-                     "merge": hbm("merge", "merge_kernel"), "multivariant": hbm("multi", "gemv_kernel (grouped)"),
+                     "merge": hbm("merge", "merge_kernel"), "multivariant_decode": hbm("multi_decode", "gemm_kernel (grouped, M=64 over 16 variants)"),
+                     "multivariant_prefill": tensor("multi_prefill", tfl_mv, "gemm_kernel (grouped, M=2112 over 16 variants)"),
                      "prefill": gemm_roof}
         dominant = max(all_roofs, key=lambda k: all_roofs[k]["share_of_step"])  # the kernel the step spends most time in
         line = {
@@ -351,7 +358,8 @@ def run_ours(args):
                        "replicas": "independent per GPU, no collective"},
             "sections": {
                 "pack_GBps": round(gbs["pack"], 1), "decode_GBps": round(gbs["decode"], 1),
-                "prefill_TFLOPps": round(tfl, 1), "multivariant_GBps": round(gbs["multi"], 1),
+                "prefill_TFLOPps": round(tfl, 1), "multivariant_decode_GBps": round(gbs["multi_decode"], 1),
+                "multivariant_prefill_TFLOPps": round(tfl_mv, 1),
                 "merge_GBps": round(gbs["merge"], 1), "ms": {s: round(sec_ms[s], 4) for s in sections}},
             "roofline": dict(all_roofs[dominant], section=dominant),
             "rooflines": all_roofs,
@@ -371,7 +379,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
