@@ -376,6 +376,48 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_only(args):
+    """One kernel family on one layer shape: a few calls over rotated weight copies (more than L2 in total),
+    timed with CUDA events.  Small enough to sit under a profiler."""
+    import torch
+    from paper_2512_19720_b200 import api, synth_torch
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    d_out, d_in = (int(t) for t in args.shape.split("x"))
+    axis = ROW if args.axis == "row" else COL
+    copies = max(2, int(300e6 // (2 * d_out * d_in)) + 1)
+    layers = []
+    for c in range(copies):
+        w_b = synth_torch.gen_base(d_out, d_in, 10 + c, dev)
+        w_f = synth_torch.gen_finetuned(w_b, 100 + c)
+        mask, v_row, v_col = api.pd_pack_delta(w_f, w_b)
+        layers.append((w_b, w_f, mask, (v_row, v_col), torch.empty_like(w_b)))
+    x = synth_torch.gen_x(args.m, d_in, 5, dev)
+    y = torch.empty((args.m, d_out), dtype=torch.float16, device=dev)
+
+    def call(i):
+        w_b, w_f, mask, v, out = layers[i % copies]
+        if args.only == "linear":
+            api.pd_linear(x, w_b, mask, v[axis], axis, y=y)
+        elif args.only == "pack":
+            api.pd_pack_delta(w_f, w_b, mask=mask, v_row=v[0], v_col=v[1])
+        else:
+            api.pd_merge(w_b, mask, v[axis], axis, w_hat=out)
+
+    call(0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.calls):
+        call(i + 1)
+    e1.record()
+    torch.cuda.synchronize()
+    if api.pd_device_status() != 0:
+        raise RuntimeError("device status latched an error")
+    print(json.dumps({"only": args.only, "shape": [d_out, d_in], "m": args.m, "axis": args.axis, "calls": args.calls,
+                      "ms_per_call_incl_launch": round(e0.elapsed_time(e1) / args.calls, 5)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -383,8 +425,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", choices=["linear", "pack", "merge"], help="run one kernel family on one layer (for profiling)")
+    ap.add_argument("--shape", default="4096x4096")
+    ap.add_argument("--m", type=int, default=16)
+    ap.add_argument("--axis", default="row", choices=["row", "col"])
+    ap.add_argument("--calls", type=int, default=4)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only:
+        run_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
