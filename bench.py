@@ -156,6 +156,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (every rank gets the result): the time of a
+    multi-GPU step is the slowest rank's.  Uses the default process group (nccl on GPUs, gloo in the CPU tests)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 # --------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -310,10 +321,7 @@ def run_ours(args):
     e2e_ms = e0.elapsed_time(e1) / args.steps
 
     # ---- max over ranks
-    stats = torch.tensor([total_ms, e2e_ms] + [sec_ms[s] for s in sections], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-    stats = stats.tolist()
+    stats = max_over_ranks([total_ms, e2e_ms] + [sec_ms[s] for s in sections], world, dev)
     total_ms, e2e_ms = stats[0], stats[1]
     sec_ms = dict(zip(sections, stats[2:]))
 
