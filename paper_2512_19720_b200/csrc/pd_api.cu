@@ -20,51 +20,75 @@ constexpr int kGroupThreads = 1024;
 //   [768, 768 + 4*M)        row_index
 constexpr size_t kOffsetsBytes = 512;
 
+// Stable counting sort of the row indices by variant id, one CTA.  Warp w owns the contiguous rows
+// [w*seg, (w+1)*seg): it counts its rows per bucket, the CTA turns the counts into start positions (bucket
+// major, warp minor), and every warp places its rows in order.  Bucket V holds the rows with id -1.
 __global__ void __launch_bounds__(kGroupThreads)
 group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict__ offsets,
                   int *__restrict__ row_index, uint32_t *__restrict__ status, int4 *__restrict__ tile_table,
                   int *__restrict__ n_token_tiles) {
-    __shared__ int warp_sums[kGroupThreads / 32];
-    __shared__ int s_base;
+    constexpr int kWarps = kGroupThreads / 32;
+    __shared__ int cnt[kWarps][kMaxVariants + 1];  // rows of warp w in bucket g, then that pair's first position
+    __shared__ int start[kMaxVariants + 2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-        s_base = 0;
-        offsets[0] = 0;
-    }
-    for (int i = threadIdx.x; i < M; i += kGroupThreads) {
-        const int id = ids[i];
-        if (id < -1 || id >= V) latch_error(status, PD_ERR_BAD_VARIANT, static_cast<uint32_t>(i));
+    const unsigned lt = (1u << lane) - 1u;
+    for (int i = threadIdx.x; i < kWarps * (kMaxVariants + 1); i += kGroupThreads) (&cnt[0][0])[i] = 0;
+    __syncthreads();
+    const int seg = (M + kWarps - 1) / kWarps;
+    const int r0 = warp * seg, r1 = min(M, r0 + seg);
+    for (int c = r0; c < r1; c += 32) {
+        const int i = c + lane;
+        int g = -2;  // -2: no row / invalid id
+        if (i < r1) {
+            const int id = ids[i];
+            if (id < -1 || id >= V) latch_error(status, PD_ERR_BAD_VARIANT, static_cast<uint32_t>(i));
+            else g = id < 0 ? V : id;
+        }
+        const unsigned same = __match_any_sync(0xffffffffu, g);
+        if (g >= 0 && (same & lt) == 0) cnt[warp][g] += __popc(same);  // lowest lane of each bucket present
+        __syncwarp();
     }
     __syncthreads();
-    for (int grp = 0; grp <= V; ++grp) {
-        const int want = (grp == V) ? -1 : grp;
-        for (int c0 = 0; c0 < M; c0 += kGroupThreads) {
-            const int i = c0 + threadIdx.x;
-            const bool hit = i < M && ids[i] == want;
-            const unsigned ballot = __ballot_sync(0xffffffffu, hit);
-            if (lane == 0) warp_sums[warp] = __popc(ballot);
-            __syncthreads();
-            int before = 0, total = 0;
-            for (int w = 0; w < kGroupThreads / 32; ++w) {
-                const int c = warp_sums[w];
-                before += (w < warp) ? c : 0;
-                total += c;
-            }
-            const int base = s_base;
-            if (hit) row_index[base + before + __popc(ballot & ((1u << lane) - 1u))] = i;
-            __syncthreads();
-            if (threadIdx.x == 0) s_base = base + total;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) offsets[grp + 1] = s_base;
+    if (threadIdx.x <= V) {  // bucket totals
+        int t = 0;
+        for (int w = 0; w < kWarps; ++w) t += cnt[w][threadIdx.x];
+        start[threadIdx.x + 1] = t;
     }
-    if (tile_table != nullptr && threadIdx.x == 0) {
-        // cut every bucket into token tiles (thread 0 wrote the offsets itself, so it may read them back)
-        int n = 0;
-        for (int grp = 0; grp <= V; ++grp)
-            for (int first = offsets[grp]; first < offsets[grp + 1]; first += kGroupedTokenTile)
-                tile_table[n++] = make_int4(grp, first, min(kGroupedTokenTile, offsets[grp + 1] - first), 0);
-        *n_token_tiles = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        start[0] = 0;
+        for (int g = 0; g <= V; ++g) start[g + 1] += start[g];
+        for (int g = 0; g <= V + 1; ++g) offsets[g] = start[g];
+        if (tile_table != nullptr) {  // cut every bucket into token tiles
+            int n = 0;
+            for (int g = 0; g <= V; ++g)
+                for (int first = start[g]; first < start[g + 1]; first += kGroupedTokenTile)
+                    tile_table[n++] = make_int4(g, first, min(kGroupedTokenTile, start[g + 1] - first), 0);
+            *n_token_tiles = n;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x <= V) {  // first position of (bucket, warp)
+        int pos = start[threadIdx.x];
+        for (int w = 0; w < kWarps; ++w) {
+            const int c = cnt[w][threadIdx.x];
+            cnt[w][threadIdx.x] = pos;
+            pos += c;
+        }
+    }
+    __syncthreads();
+    for (int c = r0; c < r1; c += 32) {
+        const int i = c + lane;
+        int g = -2;
+        if (i < r1) {
+            const int id = ids[i];
+            if (id >= -1 && id < V) g = id < 0 ? V : id;
+        }
+        const unsigned same = __match_any_sync(0xffffffffu, g);
+        if (g >= 0) row_index[cnt[warp][g] + __popc(same & lt)] = i;
+        __syncwarp();
+        if (g >= 0 && (same & lt) == 0) cnt[warp][g] += __popc(same);
+        __syncwarp();
     }
 }
 
