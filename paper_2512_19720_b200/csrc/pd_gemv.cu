@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 // tiles.  W_b and mask come from shared memory; the x fragments (and v for the col axis) are read
 // straight from global memory -- x is small and L2-resident, and keeping it out of shared memory
 // leaves the ring to the weights.  The delta term enters the same accumulator as x . (+-s) with
-// s = v[row] (row axis; exact fp16 products summed in fp32) or as (x*v) . (+-1) (col axis).
+// s = v[row] (row axis) or s = v[k] (col axis): exact fp16 products summed in fp32 either way.
 // The eight warps' partial sums are added in warp order through shared memory.
 //
 // Programmatic dependent launch: W_b and mask do not depend on the previous kernel in the stream,
@@ -378,12 +378,19 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 }
             }
             // items: (step s, block bb of this warp), k0 = s*1024 + (2*warp + bb)*64; x fragments one item ahead
-            XFrag cur, nxt;
+            // (two ahead for up to 8 tokens, where the registers allow it: the loads come from L2, ~1 us away under load)
+            constexpr int kAhead = M16 ? 1 : 2;
+            XFrag cur, nxt, nxt2;
             if (item_k0(0) < a.d_in) load_xfrag<kCol, M16>(cur, a, item_k0(0), g, t);
+            if (kAhead == 2 && 1 < n_items && item_k0(1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(1), g, t);
             for (int it = 0; it < n_items && ok; ++it) {
                 const int bb = it & 1, st = gs % kStreamStages;
                 const int k0 = item_k0(it);
-                if (it + 1 < n_items && item_k0(it + 1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(it + 1), g, t);
+                if (kAhead == 1) {
+                    if (it + 1 < n_items && item_k0(it + 1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(it + 1), g, t);
+                } else {
+                    if (it + 2 < n_items && item_k0(it + 2) < a.d_in) load_xfrag<kCol, M16>(nxt2, a, item_k0(it + 2), g, t);
+                }
                 if (bb == 0 && !(ok = mbar_wait(full + st, (gs / kStreamStages) & 1, abort_flag, a.status, 12))) break;
                 if (k0 < a.d_in) {  // else past the end of d_in: W was zero-filled there and x must not be read
                     const int blk = 2 * warp + bb;                       // block inside the step
@@ -403,11 +410,14 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         const uint32_t in_row = static_cast<uint32_t>(bi * 128) +
                                                 ((static_cast<uint32_t>(t + 4 * c) ^ static_cast<uint32_t>(((g & 1) << 2) | bi)) << 4);
                         const uint4 xa = cur.a[c], xb = cur.b[c];
-                        uint4 da = xa, db = xb;
-                        if (kCol) {
-                            const uint4 vv = cur.v[c];
-                            da = make_uint4(hmul2_u32(xa.x, vv.x), hmul2_u32(xa.y, vv.y), hmul2_u32(xa.z, vv.z), hmul2_u32(xa.w, vv.w));
-                            if (M16) db = make_uint4(hmul2_u32(xb.x, vv.x), hmul2_u32(xb.y, vv.y), hmul2_u32(xb.z, vv.z), hmul2_u32(xb.w, vv.w));
+                        // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis)
+                        uint32_t mg[2][4];
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            mg[j][0] = kCol ? cur.v[c].x : mag[j];
+                            mg[j][1] = kCol ? cur.v[c].y : mag[j];
+                            mg[j][2] = kCol ? cur.v[c].z : mag[j];
+                            mg[j][3] = kCol ? cur.v[c].w : mag[j];
                         }
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
@@ -421,9 +431,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 uint32_t pm[4];
 #pragma unroll
                                 for (int r = 0; r < 4; ++r)
-                                    pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mag[j]);
-                                mma16816(acc[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
-                                mma16816(acc[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
+                                    pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mg[j][r]);
+                                mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm[0], pm[1]);
+                                mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm[2], pm[3]);
                             }
                         }
                     }
@@ -434,6 +444,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     ++gs;
                 }
                 cur = nxt;
+                if (kAhead == 2) nxt = nxt2;
             }
 
             // ---- add the eight warps' partial sums in warp order.  The first barrier ORs "a wait ran out"
