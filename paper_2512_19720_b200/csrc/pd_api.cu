@@ -26,7 +26,7 @@ constexpr size_t kOffsetsBytes = 512;
 __global__ void __launch_bounds__(kGroupThreads)
 group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict__ offsets,
                   int *__restrict__ row_index, uint32_t *__restrict__ status, int4 *__restrict__ tile_table,
-                  int *__restrict__ n_token_tiles) {
+                  int *__restrict__ n_token_tiles, int token_tile) {
     constexpr int kWarps = kGroupThreads / 32;
     __shared__ int cnt[kWarps][kMaxVariants + 1];  // rows of warp w in bucket g, then that pair's first position
     __shared__ int start[kMaxVariants + 2];
@@ -62,8 +62,8 @@ group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict
         if (tile_table != nullptr) {  // cut every bucket into token tiles
             int n = 0;
             for (int g = 0; g <= V; ++g)
-                for (int first = start[g]; first < start[g + 1]; first += kGroupedTokenTile)
-                    tile_table[n++] = make_int4(g, first, min(kGroupedTokenTile, start[g + 1] - first), 0);
+                for (int first = start[g]; first < start[g + 1]; first += token_tile)
+                    tile_table[n++] = make_int4(g, first, min(token_tile, start[g + 1] - first), 0);
             *n_token_tiles = n;
         }
     }
@@ -115,9 +115,10 @@ pd_status check_matrix_args(const void *x, int64_t M, int64_t ldx, const void *w
 }  // namespace
 
 pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,
-                            int4 *tile_table, int *n_token_tiles, const __half *x, int64_t ldx, int64_t d_in,
-                            __half *x_sorted, cudaStream_t stream) {
-    group_rows_kernel<<<1, kGroupThreads, 0, stream>>>(ids, M, V, offsets, row_index, status, tile_table, n_token_tiles);
+                            int4 *tile_table, int *n_token_tiles, int token_tile, const __half *x, int64_t ldx,
+                            int64_t d_in, __half *x_sorted, cudaStream_t stream) {
+    group_rows_kernel<<<1, kGroupThreads, 0, stream>>>(ids, M, V, offsets, row_index, status, tile_table, n_token_tiles,
+                                                       token_tile);
     count_launch();
     if (x_sorted != nullptr) {
         const int vec_per_row = static_cast<int>(d_in / 8);
@@ -131,7 +132,7 @@ pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int 
 
 // workspace of pd_linear_multivariant beyond the status words, offsets and row index (tensor-core path only)
 size_t grouped_table_bytes(int64_t M, int32_t V) {
-    const size_t max_tiles = static_cast<size_t>(M / kGroupedTokenTile + V + 2);
+    const size_t max_tiles = static_cast<size_t>(M / kGroupedMinTokenTile + V + 2);
     return round_up(max_tiles * sizeof(int4), 256) + 256;  // tile table + the tile count
 }
 
@@ -259,14 +260,15 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
         unsigned long long col_bits = 0;
         for (int g = 0; g < V; ++g)
             if (axes[g] == PD_AXIS_COL) col_bits |= 1ull << g;
-        st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, tile_table, n_token_tiles, xh,
-                               ldx, d_in, x_sorted, stream);
+        st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, tile_table, n_token_tiles,
+                               grouped_token_tile(M, V), xh, ldx, d_in, x_sorted, stream);
         if (st != PD_OK) return st;
         return launch_gemm_grouped(x_sorted, M, static_cast<const __half *>(w_b), masks, mask_words, vh, v_stride, col_bits,
                                    V, d_out, d_in, static_cast<__half *>(y), ldy, tile_table, n_token_tiles,
-                                   static_cast<int>(M / kGroupedTokenTile + V + 2), row_index, status, stream);
+                                   static_cast<int>(M / grouped_token_tile(M, V) + V + 2), grouped_token_tile(M, V), row_index, status,
+                                   stream);
     }
-    st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, nullptr, nullptr, nullptr, 0, 0,
+    st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, nullptr, nullptr, 0, nullptr, 0, 0,
                            nullptr, stream);
     if (st != PD_OK) return st;
     for (int g = 0; g <= V; ++g) {

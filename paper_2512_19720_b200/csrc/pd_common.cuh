@@ -54,20 +54,25 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
                       uint32_t *status, cudaStream_t stream);
 
 // Multi-variant prefill: x_sorted holds the token rows in bucket order (contiguous, pitch d_in); token tile
-// i of tile_table is {variant (V = base only), first sorted row, rows (<= kGroupedTokenTile), 0}.
-constexpr int kGroupedTokenTile = 256;
+// i of tile_table is {variant (V = base only), first sorted row, rows (<= token_tile), 0}; token_tile is 64, 128
+// or 256 (grouped_token_tile picks it from the average bucket size).
+constexpr int kGroupedMinTokenTile = 64;
+inline int grouped_token_tile(int64_t M, int V) {
+    const int64_t avg = M / (V > 0 ? V : 1);
+    return avg <= 48 ? 64 : (avg <= 100 ? 128 : 256);
+}
 pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
-                              const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
-                              cudaStream_t stream);
+                              const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
+                              uint32_t *status, cudaStream_t stream);
 
 // Stable bucket sort of token rows by variant id: offsets[g] .. offsets[g+1] index row_index for
 // variant g (g = 0..V-1), offsets[V] .. offsets[V+1] the rows with id -1.  Other ids latch an error.
-// With tile_table != nullptr it also cuts every bucket into token tiles of at most kGroupedTokenTile rows
+// With tile_table != nullptr it also cuts every bucket into token tiles of at most token_tile rows
 // (tile_table, *n_token_tiles), and with x_sorted != nullptr a second kernel gathers the rows of x.
 pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int *row_index, uint32_t *status,
-                            int4 *tile_table, int *n_token_tiles, const __half *x, int64_t ldx, int64_t d_in,
-                            __half *x_sorted, cudaStream_t stream);
+                            int4 *tile_table, int *n_token_tiles, int token_tile, const __half *x, int64_t ldx,
+                            int64_t d_in, __half *x_sorted, cudaStream_t stream);
 
 }  // namespace pd

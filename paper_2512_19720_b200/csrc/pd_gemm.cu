@@ -1,21 +1,26 @@
 // Prefill path: Y[M, d_out] = X . (W_b + v (.) B)^T on the 5th-generation tensor cores.
 //
 // The MMA computes the transposed tile  D[128 output rows, BN tokens] = W_hat_tile . X_tile^T :
-//   A operand = W_hat tile, 128 rows x 64 k, K-major, 128-byte swizzle, in shared memory
+//   A operand = W_hat tile, 128 rows x 64 k, in TENSOR MEMORY (row = lane, two fp16 per 32-bit column)
 //   B operand = X tile, BN tokens x 64 k, K-major, 128-byte swizzle, in shared memory
-//   D         = fp32 accumulator in tensor memory (two buffers, so the epilogue of one
-//               tile overlaps the main loop of the next)
+//   D         = fp32 accumulator in tensor memory (256 columns)
 // Putting the weights on the 128-row side means each W_b tile is expanded once per BN = 256
-// tokens, the largest reuse one CTA can get.
+// tokens, the largest reuse one CTA can get.  Shared-memory bandwidth (TMA fills, LSU reads and
+// tensor-core operand reads share one 128 B/clk pipe) is the scarce resource: forming W_hat in
+// shared memory costs a write and a second read of every tile, forming it in tensor memory costs
+// neither.
 //
-// Pipeline per 64-wide k step (4 smem stages):
-//   producer warp   : TMA loads of the W_b tile and the X tile -> full[s]
-//   transform warps : wait full[s]; read the W_b tile from shared memory, add +-v per element
-//                     according to the mask word fetched from global memory, write it back in
-//                     place (same swizzled position), fence for the async proxy -> xform[s]
-//   MMA warp        : wait xform[s]; four tcgen05.mma (K = 16 each); commit -> empty[s]
-//   epilogue warps  : wait acc_full[b]; tcgen05.ld the 32 lanes they own, convert to fp16 and
-//                     store y[token][row]; -> acc_empty[b]
+// Three rings per 64-wide k step, decoupled so that the weights can run ahead of the MMA:
+//   x ring   (4 x 32 KB shared memory)  warp 0 : TMA load -> x_full[s];  freed by tcgen05.commit -> x_empty[s]
+//   W_b ring (4 x 16 KB shared memory)  warp 14: TMA load (+ the 64 col-axis scales) -> w_full[s];
+//                                       freed by the transform warps once the tile is in registers
+//   W_hat ring (8 x 32 TMEM columns)    transform warps: W_b row from shared memory, +-v per mask bit
+//                                       (mask words from global memory), tcgen05.st -> a_full[sa];
+//                                       freed by tcgen05.commit -> a_empty[sa]
+//   MMA warp        : wait a_full, x_full; four tcgen05.mma (K = 16 each) with A from TMEM
+//   epilogue warps  : wait acc_full; tcgen05.ld, fp16, shared-memory staging, 16-byte stores to y
+// A thread of a transform warp owns one row of the tile (its TMEM lane) and all 64 k of a step; four
+// warps take the even steps, four the odd ones.
 // Every wait is bounded; a wait that runs out latches PD_ERR_DEVICE_TIMEOUT and the CTA
 // drains and exits.
 #include "pd_ptx.cuh"
@@ -25,12 +30,13 @@ namespace {
 
 constexpr int BM = 128;          // output rows per tile (MMA M)
 constexpr int BK = 64;           // k per stage: 128 bytes of fp16 = one swizzle atom
-constexpr int kStages = 4;
+constexpr int kStages = 4;        // x ring and W_b ring (shared memory)
+constexpr int kASlots = 8;        // W_hat ring (tensor memory, 32 columns each)
 constexpr int kAccCols = 256;    // TMEM columns of the accumulator (one buffer)
 constexpr int kAccBufs = 1;
 constexpr int kACol0 = kAccBufs * kAccCols;  // first TMEM column of the W_hat ring: kStages slots of 32 columns
 constexpr int kVSlotBytes = 128;             // col axis: the 64 scales of a k step
-constexpr int kNumWarps = 14;    // 0 producer, 1 MMA, 2-5 epilogue, 6-13 transform
+constexpr int kNumWarps = 15;    // 0 x producer, 1 MMA, 2-5 epilogue, 6-13 transform, 14 W_b producer
 constexpr int kNumThreads = kNumWarps * 32;
 constexpr int kXformWarps = 8;
 constexpr int kEpiWarps = 4;
@@ -162,9 +168,10 @@ template <int BN>
 struct SmemLayout {
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
     static constexpr int kXBytes = BN * BK * 2;   // 32 KB for BN = 256
-    static constexpr int kStageBytes = kWBytes + kXBytes;
-    static constexpr int kBarOffset = kStages * kStageBytes;
-    static constexpr int kVOffset = kBarOffset + 256;        // kStages slots of kVSlotBytes
+    static constexpr int kXOffset = 0;                       // x ring
+    static constexpr int kWOffset = kStages * kXBytes;       // W_b ring
+    static constexpr int kBarOffset = kWOffset + kStages * kWBytes;
+    static constexpr int kVOffset = kBarOffset + 512;        // kStages slots of kVSlotBytes
     static constexpr int kOutOffset = kVOffset + kStages * kVSlotBytes;   // epilogue staging: [128 tokens][128 rows] fp16
     static constexpr int kTotal = kOutOffset + 128 * 128 * 2 + 1024;      // + slack for 1024-byte alignment
 };
@@ -176,9 +183,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
-    uint64_t *full = bars, *xform = bars + kStages, *empty = bars + 2 * kStages;
-    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = bars + 3 * kStages + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * kStages + 4);
+    uint64_t *x_full = bars, *x_empty = bars + kStages, *w_full = bars + 2 * kStages, *w_empty = bars + 3 * kStages;
+    uint64_t *a_full = bars + 4 * kStages, *a_empty = a_full + kASlots;
+    uint64_t *acc_full = a_empty + kASlots, *acc_empty = acc_full + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
+    static_assert((4 * kStages + 2 * kASlots + 2) * 8 + 8 <= 512, "barrier block");
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -187,9 +196,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full + s, 1);
-            mbar_init(xform + s, kXformWarps / 2);  // the four warps (one per TMEM lane quarter) that own the stage
-            mbar_init(empty + s, 1);
+            mbar_init(x_full + s, 1);
+            mbar_init(x_empty + s, 1);
+            mbar_init(w_full + s, 1);
+            mbar_init(w_empty + s, kXformWarps / 2);  // the four warps (one per TMEM lane quarter) that own the stage
+        }
+        for (int s = 0; s < kASlots; ++s) {
+            mbar_init(a_full + s, kXformWarps / 2);
+            mbar_init(a_empty + s, 1);
         }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(acc_full + b, 1);
@@ -208,32 +222,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
-        // ------------------------------------------------ TMA producer
+    if (warp == 0 || warp == kNumWarps - 1) {
+        // ------------------------------------------------ TMA producers: warp 0 feeds the x ring, the last warp the W_b ring
         if (lane == 0) {
+            const bool is_x = warp == 0;
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                     const int s = it % kStages;
-                    if (!(ok = mbar_wait(empty + s, ((it / kStages) & 1) ^ 1, abort_flag, a.status, 1))) break;
-                    unsigned char *st = smem + s * L::kStageBytes;
-                    const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
-                    mbar_arrive_expect_tx(full + s, L::kStageBytes + v_bytes);
-                    tma_load_2d(&map_w, full + s, st, ks * BK, ti.tm * BM);
-                    tma_load_2d(&map_x, full + s, st + L::kWBytes, ks * BK, ti.tok0);
-                    if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, full + s);
+                    const uint32_t parity = ((it / kStages) & 1) ^ 1;
+                    if (is_x) {
+                        if (!(ok = mbar_wait(x_empty + s, parity, abort_flag, a.status, 1))) break;
+                        mbar_arrive_expect_tx(x_full + s, L::kXBytes);
+                        tma_load_2d(&map_x, x_full + s, smem + L::kXOffset + s * L::kXBytes, ks * BK, ti.tok0);
+                    } else {
+                        if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
+                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
+                        mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
+                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, ti.tm * BM);
+                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
+        // ------------------------------------------------ MMA issuer: A = W_hat slot in tensor memory, B = x tile in shared memory
         if (lane == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
-                // MMA N = the tile's tokens rounded up to 16 (the whole 256-token box in the plain mode)
+                // MMA N = the tile's tokens rounded up to 16 (the whole token box in the plain mode)
                 const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
                 const int n_mma = GROUPED ? ((ti.count + 15) & ~15) : BN;
                 const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
@@ -242,20 +262,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + b * kAccCols;
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
-                    const int s = it % kStages;
-                    if (!(ok = mbar_wait(xform + s, (it / kStages) & 1, abort_flag, a.status, 3))) break;
+                    const int s = it % kStages, sa = it % kASlots;
+                    if (!(ok = mbar_wait(a_full + sa, (it / kASlots) & 1, abort_flag, a.status, 3))) break;
+                    if (!(ok = mbar_wait(x_full + s, (it / kStages) & 1, abort_flag, a.status, 7))) break;
                     tcgen05_fence_after();
-                    const uint32_t w_addr = smem_u32(smem + s * L::kStageBytes);
-                    const uint32_t x_addr = w_addr + L::kWBytes;
+                    const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kXBytes);
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) {
-                        const uint64_t db = make_smem_desc(x_addr + kk * 32);
-                        if (ti.delta)  // A = the W_hat slot the transform warps filled in tensor memory
-                            tcgen05_mma_f16_tmem_a(d_tmem, tmem_base + kACol0 + s * 32 + kk * 8, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-                        else           // base only: A = the W_b tile as TMA delivered it
-                            tcgen05_mma_f16(d_tmem, make_smem_desc(w_addr + kk * 32), db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-                    }
-                    tcgen05_commit(empty + s);  // frees the stage when these MMAs have read it
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tcgen05_mma_f16_tmem_a(d_tmem, tmem_base + kACol0 + sa * 32 + kk * 8, make_smem_desc(x_addr + kk * 32), idesc,
+                                               (ks > 0 || kk > 0) ? 1u : 0u);
+                    tcgen05_commit(x_empty + s);   // both free up when these MMAs have read their operands
+                    tcgen05_commit(a_empty + sa);
                 }
                 if (ok) tcgen05_commit(acc_full + b);
             }
@@ -357,18 +374,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             load_words(ks, wn0, wn1);
             for (; ks < a.k_steps; ks += 2) {
                 const uint32_t my_it = it + ks;
-                const int s = my_it % kStages;
+                const int s = my_it % kStages, sa = my_it % kASlots;
                 const uint32_t word[2] = {wn0, wn1};
                 load_words(ks + 2, wn0, wn1);
                 // the TMEM store below is warp-collective: all lanes leave together or not at all
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(full + s, (my_it / kStages) & 1, abort_flag, a.status, 5)))) break;
-                if (delta) {
-                    const unsigned char *wt = smem + s * L::kStageBytes + r * 128;
-                    const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
-                    uint32_t out[32];
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, (my_it / kStages) & 1, abort_flag, a.status, 5)))) break;
+                const unsigned char *wt = smem + L::kWOffset + s * L::kWBytes + r * 128;
+                const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
+                uint32_t out[32];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {  // 16-byte piece c = columns 8c .. 8c+7 of the stage
-                        const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
+                for (int c = 0; c < 8; ++c) {  // 16-byte piece c = columns 8c .. 8c+7 of the stage
+                    const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
+                    const uint32_t wp[4] = {w.x, w.y, w.z, w.w};
+                    if (delta) {
                         uint32_t vv[4] = {vrow, vrow, vrow, vrow};
                         if (col) {
                             const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
@@ -377,20 +395,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                         const uint32_t bits = word[c >> 2];
                         const int j = c & 3;  // byte of the word that belongs to this piece
                         const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
-                        const uint32_t wp[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
                         for (int pr = 0; pr < 4; ++pr) {
                             // halves 2pr (low) and 2pr+1 (high) of the piece: +v where the bit is 1, -v where it is 0
                             const uint32_t rep = prmt(bits << (7 - 2 * pr), bits << (6 - 2 * pr), sel);
                             out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
                         }
+                    } else {  // base only: the tile goes to tensor memory unchanged
+#pragma unroll
+                        for (int pr = 0; pr < 4; ++pr) out[4 * c + pr] = wp[pr];
                     }
-                    tcgen05_st_32x32b_x32(a_taddr + s * 32, out);
-                    tcgen05_wait_st();
-                    tcgen05_fence_before();
                 }
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(a_empty + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
+                tcgen05_fence_after();
+                tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
+                // The store takes every register of the tile row as an operand, so all shared-memory reads of the
+                // W_b slot have returned by now: only here may the slot be handed back for refilling.
                 __syncwarp();
-                if (lane == 0) mbar_arrive(xform + s);
+                if (lane == 0) mbar_arrive(w_empty + s);
+                tcgen05_wait_st();
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full + sa);
             }
             it += a.k_steps;
         }
@@ -485,12 +511,14 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
     return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
 }
 
-pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
+namespace {
+
+template <int BN>
+pd_status launch_gemm_grouped_bn(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
                               cudaStream_t stream) {
-    constexpr int BN = kGroupedTokenTile;
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, BN)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -516,6 +544,22 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
     const int64_t tiles = static_cast<int64_t>(args.tiles_m) * max_token_tiles;  // upper bound; the kernel reads the real count
     const int grid = tiles < sm_count() ? static_cast<int>(tiles) : sm_count();
     return launch_one<PD_AXIS_ROW, true, true, BN>(mw, mx, args, grid, stream);
+}
+
+}  // namespace
+
+pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
+                              int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
+                              int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
+                              const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
+                              uint32_t *status, cudaStream_t stream) {
+#define PD_GROUPED(BN)                                                                                                     \
+    return launch_gemm_grouped_bn<BN>(x_sorted, M, w_b, masks, mask_stride, vs, v_stride, col_axis_bits, V, d_out, d_in, y, \
+                                      ldy, tile_table, n_token_tiles, max_token_tiles, row_index, status, stream)
+    if (token_tile == 64) PD_GROUPED(64);
+    if (token_tile == 128) PD_GROUPED(128);
+    PD_GROUPED(256);
+#undef PD_GROUPED
 }
 
 }  // namespace pd
