@@ -11,13 +11,15 @@
 // neither.
 //
 // Three rings per 64-wide k step, decoupled so that the weights can run ahead of the MMA:
-//   x ring   (4 x 32 KB shared memory)  warp 0 : TMA load -> x_full[s];  freed by tcgen05.commit -> x_empty[s]
-//   W_b ring (4 x 16 KB shared memory)  warp 14: TMA load (+ the 64 col-axis scales) -> w_full[s];
-//                                       freed by the transform warps once the tile is in registers
-//   W_hat ring (8 x 32 TMEM columns)    transform warps: W_b row from shared memory, +-v per mask bit
-//                                       (mask words from global memory), tcgen05.st -> a_full[sa];
-//                                       freed by tcgen05.commit -> a_empty[sa]
-//   MMA warp        : wait a_full, x_full; four tcgen05.mma (K = 16 each) with A from TMEM
+//   x ring   (4..8 slots, shared memory)  warp 0 : TMA load of the x tile, signalled on ready[it % 8]
+//   W_b ring (4..8 x 16 KB shared memory) warp 14: TMA load (+ the 64 col-axis scales) -> w_full[s];
+//                                         freed by the transform warps once the tile row is in TMEM
+//   W_hat ring (8 x 32 TMEM columns)      transform warps: W_b row from shared memory, +-v per mask bit
+//                                         (mask words from global memory), tcgen05.st, arrive on ready[it % 8]
+//   MMA warp        : ONE wait per k step (ready: x landed and W_hat written), four tcgen05.mma (K = 16 each)
+//                     with A from TMEM, ONE tcgen05.commit -> consumed[it % 8], which frees the x slot (producer)
+//                     and the W_hat slot (transform warps).  The issuing thread costs ~70 clocks per MMA or commit
+//                     and ~100 per wait; with two waits and two commits it was slower than the tensor core.
 //   epilogue warps  : wait acc_full; tcgen05.ld, fp16, shared-memory staging, 16-byte stores to y
 // A thread of a transform warp owns one row of the tile (its TMEM lane) and all 64 k of a step; four
 // warps take the even steps, four the odd ones.
@@ -30,11 +32,11 @@ namespace {
 
 constexpr int BM = 128;          // output rows per tile (MMA M)
 constexpr int BK = 64;           // k per stage: 128 bytes of fp16 = one swizzle atom
-constexpr int kStages = 4;        // x ring and W_b ring (shared memory)
+constexpr int kMaxStages = 8;      // the x ring has SmemLayout<BN>::kXStages slots, the W_b ring ::kWStages
 constexpr int kASlots = 8;        // W_hat ring (tensor memory, 32 columns each)
 constexpr int kAccCols = 256;    // TMEM columns of the accumulator (one buffer)
 constexpr int kAccBufs = 1;
-constexpr int kACol0 = kAccBufs * kAccCols;  // first TMEM column of the W_hat ring: kStages slots of 32 columns
+constexpr int kACol0 = kAccBufs * kAccCols;  // first TMEM column of the W_hat ring: kASlots slots of 32 columns
 constexpr int kVSlotBytes = 128;             // col axis: the 64 scales of a k step
 constexpr int kNumWarps = 15;    // 0 x producer, 1 MMA, 2-5 epilogue, 6-13 transform, 14 W_b producer
 constexpr int kNumThreads = kNumWarps * 32;
@@ -169,12 +171,48 @@ struct SmemLayout {
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
     static constexpr int kXBytes = BN * BK * 2;   // 32 KB for BN = 256
     static constexpr int kXOffset = 0;                       // x ring
-    static constexpr int kWOffset = kStages * kXBytes;       // W_b ring
-    static constexpr int kBarOffset = kWOffset + kStages * kWBytes;
-    static constexpr int kVOffset = kBarOffset + 512;        // kStages slots of kVSlotBytes
-    static constexpr int kOutOffset = kVOffset + kStages * kVSlotBytes;   // epilogue staging: [128 tokens][128 rows] fp16
+    // W_b ring: what a narrow x tile leaves free goes to more W_b stages -- with few tokens per tile a k step is
+    // short and only a deep ring hides the L2/HBM latency of the weight tiles
+    static constexpr int kWStages = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int kXStages = kWStages;
+    static constexpr int kWOffset = kXStages * kXBytes;
+    static constexpr int kBarOffset = kWOffset + kWStages * kWBytes;
+    static constexpr int kVOffset = kBarOffset + 512;        // kWStages slots of kVSlotBytes
+    static constexpr int kOutOffset = kVOffset + kWStages * kVSlotBytes;   // epilogue staging: [128 tokens][128 rows] fp16
+    static_assert(kWStages % 2 == 0 && kWStages <= kMaxStages, "even and odd k steps belong to different warps");
     static constexpr int kTotal = kOutOffset + 128 * 128 * 2 + 1024;      // + slack for 1024-byte alignment
 };
+
+// One row of a W_hat tile: 64 columns = 8 pieces of 16 bytes read from the 128-byte-swizzled W_b tile, +-v added
+// per mask bit (word0 = columns 0..31, word1 = columns 32..63), packed two fp16 per register in column order.
+template <bool DELTA, bool COL>
+__device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsigned char *wt, const unsigned char *vs, int r,
+                                                uint32_t vrow, uint32_t word0, uint32_t word1) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {  // 16-byte piece c = columns 8c .. 8c+7 of the stage
+        const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
+        const uint32_t wp[4] = {w.x, w.y, w.z, w.w};
+        if (DELTA) {
+            uint32_t vv[4] = {vrow, vrow, vrow, vrow};
+            if (COL) {
+                const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
+                vv[0] = t4.x, vv[1] = t4.y, vv[2] = t4.z, vv[3] = t4.w;
+            }
+            const uint32_t bits = c < 4 ? word0 : word1;
+            const int j = c & 3;  // byte of the word that belongs to this piece
+            const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
+#pragma unroll
+            for (int pr = 0; pr < 4; ++pr) {
+                // halves 2pr (low) and 2pr+1 (high) of the piece: +v where the bit is 1, -v where it is 0
+                const uint32_t rep = prmt(bits << (7 - 2 * pr), bits << (6 - 2 * pr), sel);
+                out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
+            }
+        } else {  // base only: the tile goes to tensor memory unchanged
+#pragma unroll
+            for (int pr = 0; pr < 4; ++pr) out[4 * c + pr] = wp[pr];
+        }
+    }
+}
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
 __global__ void __launch_bounds__(kNumThreads, 1)
@@ -183,11 +221,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
-    uint64_t *x_full = bars, *x_empty = bars + kStages, *w_full = bars + 2 * kStages, *w_empty = bars + 3 * kStages;
-    uint64_t *a_full = bars + 4 * kStages, *a_empty = a_full + kASlots;
-    uint64_t *acc_full = a_empty + kASlots, *acc_empty = acc_full + 1;
+    // ready[it % 8]   : k step `it` can be multiplied -- its x tile has landed (TMA bytes + the producer's arrival)
+    //                   and its W_hat slot is written (four transform warps);
+    // consumed[it % 8]: the MMAs of k step `it` have finished reading both (tcgen05.commit).
+    // One wait and one commit per k step keep the single MMA-issuing thread ahead of the tensor core.
+    uint64_t *w_full = bars, *w_empty = bars + kMaxStages;
+    uint64_t *ready = bars + 2 * kMaxStages, *consumed = ready + kASlots;
+    uint64_t *acc_full = consumed + kASlots, *acc_empty = acc_full + 1;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
-    static_assert((4 * kStages + 2 * kASlots + 2) * 8 + 8 <= 512, "barrier block");
+    static_assert((2 * kMaxStages + 2 * kASlots + 2) * 8 + 8 <= 512, "barrier block");
+    static_assert(L::kXStages <= kASlots, "an x slot must be free again before its ready barrier comes round");
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -195,15 +238,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     const int n_tiles = a.tiles_m * n_tt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(x_full + s, 1);
-            mbar_init(x_empty + s, 1);
+        for (int s = 0; s < L::kWStages; ++s) {
             mbar_init(w_full + s, 1);
             mbar_init(w_empty + s, kXformWarps / 2);  // the four warps (one per TMEM lane quarter) that own the stage
         }
         for (int s = 0; s < kASlots; ++s) {
-            mbar_init(a_full + s, kXformWarps / 2);
-            mbar_init(a_empty + s, 1);
+            mbar_init(ready + s, kXformWarps / 2 + 1);
+            mbar_init(consumed + s, 1);
         }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(acc_full + b, 1);
@@ -212,7 +253,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (threadIdx.x < kStages * kVSlotBytes / 4) {  // scale slots start at zero: a short last k step leaves its tail untouched
+    if (threadIdx.x < L::kWStages * kVSlotBytes / 4) {  // scale slots start at zero: a short last k step leaves its tail untouched
         reinterpret_cast<uint32_t *>(smem + L::kVOffset)[threadIdx.x] = 0u;
         fence_proxy_async_smem();
     }
@@ -231,12 +272,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t parity = ((it / kStages) & 1) ^ 1;
+                    const int ring = is_x ? L::kXStages : L::kWStages;
+                    const int s = it % ring;
+                    const uint32_t parity = ((it / ring) & 1) ^ 1;
                     if (is_x) {
-                        if (!(ok = mbar_wait(x_empty + s, parity, abort_flag, a.status, 1))) break;
-                        mbar_arrive_expect_tx(x_full + s, L::kXBytes);
-                        tma_load_2d(&map_x, x_full + s, smem + L::kXOffset + s * L::kXBytes, ks * BK, ti.tok0);
+                        // the x slot was last read by k step it - kXStages
+                        if (it >= static_cast<uint32_t>(L::kXStages)) {
+                            const uint32_t prev = it - L::kXStages;
+                            if (!(ok = mbar_wait(consumed + prev % kASlots, (prev / kASlots) & 1, abort_flag, a.status, 1))) break;
+                        }
+                        mbar_arrive_expect_tx(ready + it % kASlots, L::kXBytes);
+                        tma_load_2d(&map_x, ready + it % kASlots, smem + L::kXOffset + s * L::kXBytes, ks * BK, ti.tok0);
                     } else {
                         if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
                         const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
@@ -262,17 +308,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + b * kAccCols;
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
-                    const int s = it % kStages, sa = it % kASlots;
-                    if (!(ok = mbar_wait(a_full + sa, (it / kASlots) & 1, abort_flag, a.status, 3))) break;
-                    if (!(ok = mbar_wait(x_full + s, (it / kStages) & 1, abort_flag, a.status, 7))) break;
+                    const int s = it % L::kXStages, sa = it % kASlots;
+                    if (!(ok = mbar_wait(ready + sa, (it / kASlots) & 1, abort_flag, a.status, 3))) break;
                     tcgen05_fence_after();
                     const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kXBytes);
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; ++kk)
                         tcgen05_mma_f16_tmem_a(d_tmem, tmem_base + kACol0 + sa * 32 + kk * 8, make_smem_desc(x_addr + kk * 32), idesc,
                                                (ks > 0 || kk > 0) ? 1u : 0u);
-                    tcgen05_commit(x_empty + s);   // both free up when these MMAs have read their operands
-                    tcgen05_commit(a_empty + sa);
+                    tcgen05_commit(consumed + sa);  // the x slot and the W_hat slot free up when these MMAs have read them
                 }
                 if (ok) tcgen05_commit(acc_full + b);
             }
@@ -370,43 +414,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
             };
             int ks = static_cast<int>((par ^ it) & 1u);  // first k step of this tile that falls to this warp
-            uint32_t wn0, wn1;
-            load_words(ks, wn0, wn1);
+            // mask words of the next four k steps of this warp, in flight: they come from L2 or HBM, and with few
+            // tokens per tile a k step is far shorter than that latency
+            uint32_t q0[4], q1[4];
+#pragma unroll
+            for (int d = 0; d < 4; ++d) load_words(ks + 2 * d, q0[d], q1[d]);
             for (; ks < a.k_steps; ks += 2) {
                 const uint32_t my_it = it + ks;
-                const int s = my_it % kStages, sa = my_it % kASlots;
-                const uint32_t word[2] = {wn0, wn1};
-                load_words(ks + 2, wn0, wn1);
+                const int s = my_it % L::kWStages, sa = my_it % kASlots;
+                const uint32_t word[2] = {q0[0], q1[0]};
+#pragma unroll
+                for (int d = 0; d < 3; ++d) q0[d] = q0[d + 1], q1[d] = q1[d + 1];
+                load_words(ks + 8, q0[3], q1[3]);
                 // the TMEM store below is warp-collective: all lanes leave together or not at all
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, (my_it / kStages) & 1, abort_flag, a.status, 5)))) break;
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, (my_it / L::kWStages) & 1, abort_flag, a.status, 5)))) break;
                 const unsigned char *wt = smem + L::kWOffset + s * L::kWBytes + r * 128;
                 const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
                 uint32_t out[32];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {  // 16-byte piece c = columns 8c .. 8c+7 of the stage
-                    const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
-                    const uint32_t wp[4] = {w.x, w.y, w.z, w.w};
-                    if (delta) {
-                        uint32_t vv[4] = {vrow, vrow, vrow, vrow};
-                        if (col) {
-                            const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
-                            vv[0] = t4.x, vv[1] = t4.y, vv[2] = t4.z, vv[3] = t4.w;
-                        }
-                        const uint32_t bits = word[c >> 2];
-                        const int j = c & 3;  // byte of the word that belongs to this piece
-                        const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
-#pragma unroll
-                        for (int pr = 0; pr < 4; ++pr) {
-                            // halves 2pr (low) and 2pr+1 (high) of the piece: +v where the bit is 1, -v where it is 0
-                            const uint32_t rep = prmt(bits << (7 - 2 * pr), bits << (6 - 2 * pr), sel);
-                            out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
-                        }
-                    } else {  // base only: the tile goes to tensor memory unchanged
-#pragma unroll
-                        for (int pr = 0; pr < 4; ++pr) out[4 * c + pr] = wp[pr];
-                    }
-                }
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(a_empty + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
+                // specialised bodies: with the variant known only at run time (grouped mode) a single body with
+                // the tests inside the unrolled loop spilled registers and ran four times slower
+                if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[0], word[1]);
+                else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
                 tcgen05_fence_after();
                 tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
                 // The store takes every register of the tile row as an operand, so all shared-memory reads of the
@@ -416,7 +446,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 tcgen05_wait_st();
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(a_full + sa);
+                if (lane == 0) mbar_arrive(ready + sa);
             }
             it += a.k_steps;
         }
