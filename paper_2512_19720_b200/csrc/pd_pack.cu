@@ -51,8 +51,9 @@ __device__ __forceinline__ long long half_units(uint32_t h) {
     return (h & 0x8000u) ? -mag : mag;
 }
 
-// |a - b| in units of 2^-24 for two binary16 values both below 0.25 in magnitude: the fp32
-// difference is exact (23 bits), and adding 0.5 places it where one fp32 ulp is 2^-24.
+// |a - b| in units of 2^-24 for two binary16 values less than 0.5 apart: the fp32 difference is exact
+// (a multiple of 2^-24 below 2^23 units), and adding 0.5 places it where one fp32 ulp is 2^-24.  For
+// values 0.5 or more apart the result is >= 2^23 (or has high bits set), which the caller tests.
 __device__ __forceinline__ uint32_t abs_diff_units_small(float a, float b) {
     return __float_as_uint(fabsf(__fsub_rn(a, b)) + 0.5f) - 0x3f000000u;
 }
@@ -85,25 +86,30 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
             const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
             const uint4 a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
             const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
-            uint32_t big = 0;
+            uint32_t spread = 0, u[8], u_or = 0;
 #pragma unroll
             for (int p = 0; p < 4; ++p) {
-                // bit = (w_f >= w_b): exact on binary16, false for NaN, true for -0 vs +0
-                const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p])) & 0x00010001u;
-                bits |= ((ge | (ge >> 15)) & 3u) << (2 * p);
-                big |= ((a[p] & 0x7fff7fffu) + 0x4c004c00u) | ((b[p] & 0x7fff7fffu) + 0x4c004c00u);
+                // bit = (w_f >= w_b): exact on binary16, false for NaN, true for -0 vs +0.  The comparison gives
+                // 0xffff per true half; pair p keeps bit 2p of the low half and bit 2p+1 of the high half.
+                const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p]));
+                spread |= ge & ((1u << (2 * p)) | (1u << (17 + 2 * p)));
+                // |dW| in units of 2^-24 by the fp32 trick.  Every binary16 is a multiple of 2^-24, so whenever
+                // |dW| < 0.5 the fp32 difference is exact and |dW| + 0.5 lies in [0.5, 1), where one ulp is 2^-24.
+                const float2 fa = __half22float2(as_half2(a[p])), fb = __half22float2(as_half2(b[p]));
+                u[2 * p] = abs_diff_units_small(fa.x, fb.x);
+                u[2 * p + 1] = abs_diff_units_small(fa.y, fb.y);
+                u_or |= u[2 * p] | u[2 * p + 1];
             }
-            slow = (big & 0x80008000u) != 0;  // some |w| >= 0.25 (0x3400)
+            bits = (spread | (spread >> 16)) & 0xffu;
+            slow = (u_or & 0xff800000u) != 0;  // some |dW| >= 0.5 (or not finite): take the exact 64-bit path
             if (!slow) {
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    const float2 fa = __half22float2(as_half2(a[p])), fb = __half22float2(as_half2(b[p]));
-                    const uint32_t u0 = abs_diff_units_small(fa.x, fb.x), u1 = abs_diff_units_small(fa.y, fb.y);
                     if (COL) {
-                        cacc[2 * p] += u0;
-                        cacc[2 * p + 1] += u1;
+                        cacc[2 * p] += u[2 * p];
+                        cacc[2 * p + 1] += u[2 * p + 1];
                     }
-                    fast_sum += u0 + u1;
+                    fast_sum += u[2 * p] + u[2 * p + 1];
                 }
             } else {
 #pragma unroll
@@ -112,9 +118,9 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
                     for (int h = 0; h < 2; ++h) {
                         const long long d = half_units((a[p] >> (16 * h)) & 0xffffu) -
                                             half_units((b[p] >> (16 * h)) & 0xffffu);
-                        const unsigned long long u = static_cast<unsigned long long>(d < 0 ? -d : d);
-                        slow_sum += u;
-                        if (COL) atomicAdd(col_sum + col0 + 2 * p + h, u);
+                        const unsigned long long du = static_cast<unsigned long long>(d < 0 ? -d : d);
+                        slow_sum += du;
+                        if (COL) atomicAdd(col_sum + col0 + 2 * p + h, du);
                     }
                 }
             }
@@ -187,7 +193,7 @@ merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *
             vf[2 * p + 1] = f.y;
         }
     }
-#pragma unroll 4
+#pragma unroll 8
     for (int rr = warp; rr < kTileRows; rr += kThreads / 32) {
         const int o = row0 + rr;
         if (o >= d_out) break;
