@@ -11,7 +11,7 @@ size_t grouped_table_bytes(int64_t M, int32_t V);
 namespace {
 
 constexpr int kMaxVariants = 64;
-constexpr int kGemvMaxTokens = 64;  // up to here the decode kernel runs in chunks of 16 rows
+constexpr int kGemvMaxTokens = 16;  // above it one tensor-core launch (64-token tiles) beats several decode passes over W_b
 constexpr int kGroupThreads = 1024;
 
 // workspace layout of the linear calls:
