@@ -39,6 +39,9 @@ PREFILL_M = (256, 2048, 8192)
 N_VARIANTS = 16
 MULTI_M = (64, 64 + 4 * 512)
 ROW, COL = 0, 1
+# ncu dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, 4096 x 11008 captures in profiles/
+# (merge: reads only -- half of its writes are still dirty in L2 when the kernel ends)
+NCU_DRAM_RATIO = {"decode": 96.13 / 95.81, "pack": (180.52 + 4.84) / (180.36 + 5.67), "merge": 1.0}
 METRIC = "fused delta-linear decode HBM GB/s (7B block sweep, M in {1,4,16}, row+col axes)"
 
 
@@ -335,7 +338,11 @@ def run_ours(args):
             per_gpu = gbs[section] / world
             return {"kernel": kernel, "bound": "hbm", "achieved": round(per_gpu, 1), "peak": pk["hbm_gbs"],
                     "unit": "GB/s", "frac": round(per_gpu / pk["hbm_gbs"], 4), "frac_of": pk["source"],
-                    "frac_of_nominal_8TBs": round(per_gpu / 8000.0, 4), "traffic": None,
+                    "frac_of_nominal_8TBs": round(per_gpu / 8000.0, 4),
+                    # DRAM bytes per call = algorithmic bytes x (ncu dram bytes / algorithmic bytes) of the captured
+                    # case under profiles/ (traffic grows in proportion to the elements streamed)
+                    "traffic": (round(work[section] / calls_per[section] * NCU_DRAM_RATIO[section])
+                                if section in NCU_DRAM_RATIO else None),
                     "algorithmic_bytes_per_call": work[section] // calls_per[section],
                     "avg_call_ms": round(sec_ms[section] / calls_per[section], 5),
                     "share_of_step": round(sec_ms[section] / sum(sec_ms.values()), 4)}
