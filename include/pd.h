@@ -103,6 +103,19 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx,
                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * pd_linear_host -- pd_linear for activations that live in HOST memory (same operation and paper passages
+ * as pd_linear).  Enqueues, on cuda_stream: copy of x_host -> x_dev, the fused linear, copy of y_dev -> y_host.
+ *
+ *   x_host : in,  HOST fp16 [M, d_in], dense (row stride d_in); pinned memory makes the copies asynchronous
+ *   y_host : out, HOST fp16 [M, d_out], dense
+ *   x_dev, y_dev : device staging buffers owned by the caller, at least M*d_in and M*d_out fp16, 16-byte aligned
+ *   everything else as in pd_linear.  The results are in y_host once the stream has been synchronised.
+ */
+pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void *w_b, const uint32_t *mask,
+                         const void *v, pd_axis axis, int64_t d_out, int64_t d_in, void *y_dev, void *y_host,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * pd_linear_multivariant -- one batch, many fine-tunes over one base.
  * Paper: Method section ("multiple fine-tuned models ... all share the same underlying base
  * weights"); the per-row routing is this library's reading of multi-tenant serving.

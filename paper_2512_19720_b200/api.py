@@ -18,7 +18,7 @@ OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE = 0, 1, 2, 3
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpd.so")
 
-EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
+EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
            "pd_device_status", "pd_status_string", "pd_launch_count"]
 
 
@@ -40,6 +40,8 @@ def _load() -> ctypes.CDLL:
     lib.pd_pack_delta_static.restype = ctypes.c_int
     lib.pd_linear.argtypes = [p, i64, i64, p, p, p, ctypes.c_int, i64, i64, p, i64, p, sz, p]
     lib.pd_linear.restype = ctypes.c_int
+    lib.pd_linear_host.argtypes = [p, p, i64, p, p, p, ctypes.c_int, i64, i64, p, p, p, sz, p]
+    lib.pd_linear_host.restype = ctypes.c_int
     lib.pd_linear_multivariant.argtypes = [p, i64, i64, p, p, p, p, i64, p, i32, i64, i64, p, i64, p, sz, p]
     lib.pd_linear_multivariant.restype = ctypes.c_int
     lib.pd_merge.argtypes = [p, p, p, ctypes.c_int, i64, i64, p, p]
@@ -148,6 +150,22 @@ def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None):
     _check(lib.pd_linear(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
                          y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pd_linear")
     return y
+
+
+def pd_linear_host(x_host, x_dev, w_b, mask, v, axis, y_dev, y_host, workspace=None):
+    """pd_linear with the activations in host memory: x_host (CPU fp16 [M, d_in], ideally pinned) is copied to the
+    staging tensor x_dev, the linear runs, y_dev is copied to y_host; all on the current stream, nothing synchronised."""
+    assert x_host.dtype == torch.float16 and y_host.dtype == torch.float16 and not x_host.is_cuda and not y_host.is_cuda
+    assert x_host.is_contiguous() and y_host.is_contiguous() and x_dev.is_contiguous() and y_dev.is_contiguous()
+    m, d_in = x_host.shape
+    d_out = w_b.shape[0]
+    assert x_dev.numel() >= m * d_in and y_dev.numel() >= m * d_out and tuple(y_host.shape) == (m, d_out)
+    need = workspace_bytes(OP_LINEAR, m, 0, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, w_b.device)
+    _check(lib.pd_linear_host(x_host.data_ptr(), _ptr(x_dev), m, _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in,
+                              _ptr(y_dev), y_host.data_ptr(), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "pd_linear_host")
+    return y_host
 
 
 def pd_linear_multivariant(x, variant_ids, w_b, masks, vs, axes, y=None, workspace=None):

@@ -226,6 +226,19 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
     return PD_OK;
 }
 
+pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void *w_b, const uint32_t *mask, const void *v,
+                         pd_axis axis, int64_t d_out, int64_t d_in, void *y_dev, void *y_host, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream) {
+    if (!x_host || !x_dev || !y_dev || !y_host || M <= 0 || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * d_in * sizeof(__half), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return PD_ERR_CUDA;
+    const pd_status st = pd_linear(x_dev, M, d_in, w_b, mask, v, axis, d_out, d_in, y_dev, d_out, workspace, workspace_bytes,
+                                   cuda_stream);
+    if (st != PD_OK) return st;
+    return cuda_ok(cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * d_out * sizeof(__half), cudaMemcpyDeviceToHost, stream));
+}
+
 pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
                                  const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes,
                                  int32_t V, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,

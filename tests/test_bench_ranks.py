@@ -26,7 +26,10 @@ def _worker(rank, world, port, out_dir):
 
 
 def test_timings_are_combined_as_max_over_ranks(tmp_path):
-    port = 29500 + os.getpid() % 2000
+    import socket
+    with socket.socket() as sock:  # a port nobody is using right now
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     for rank in range(2):
         assert json.load(open(tmp_path / f"r{rank}.json")) == [11.0, 5.0, 7.0]

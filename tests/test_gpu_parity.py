@@ -234,6 +234,32 @@ def test_linear_between_decode_and_prefill(api, m):
     check_linear(api, layer(200, 1152, seed=3), m, COL)
 
 
+def test_linear_host_buffers_side_stream_and_odd_output_pitch(api):
+    # pd_linear_host: x from pinned host memory, y back to pinned host memory, on a non-default stream
+    L = layer(1024, 1024)
+    for m in (4, 40):
+        x = synth.gen_x(m, 1024, 30 + m)
+        ref = orc.linear(x, L.w_b, L.mask, L.v_col, COL)
+        x_host = torch.from_numpy(x).pin_memory()
+        y_host = torch.empty((m, 1024), dtype=torch.float16).pin_memory()
+        x_dev = torch.empty((m, 1024), dtype=torch.float16, device="cuda")
+        y_dev = torch.empty((m, 1024), dtype=torch.float16, device="cuda")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            api.pd_linear_host(x_host, x_dev, L.d_w_b, L.d_mask, L.d_v_col, COL, y_dev, y_host)
+        side.synchronize()
+        assert rel_err(y_host.numpy(), ref) <= TOL
+        # an output view with an odd row pitch and a 2-byte-aligned base: the vector stores must not be used
+        buf = torch.zeros((m, 1024 + 3), dtype=torch.float16, device="cuda")
+        y_view = buf[:, 1:1025]
+        api.pd_linear(dev(x), L.d_w_b, L.d_mask, L.d_v_col, COL, y=y_view)
+        torch.cuda.synchronize()
+        assert api.pd_device_status() == 0
+        assert rel_err(host(y_view), ref) <= TOL
+        assert bool((buf[:, 0] == 0).all()) and bool((buf[:, 1025:] == 0).all())
+
+
 # ------------------------------------------------------------------ prefill linear (tensor-core path)
 def check_prefill(api, L, m, axis, rows=None, seed=2000):
     x = synth.gen_x(m, L.d_in, seed)
