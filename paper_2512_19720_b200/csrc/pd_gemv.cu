@@ -265,9 +265,11 @@ constexpr int kStreamConsumers = 8;
 constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
 constexpr int kStW = 0;                     // 4 boxes of [16 rows][4 blocks][128 B], swizzled (8 KB each)
 constexpr int kStMask = 32768;              // [16 rows][32 words]
-constexpr int kStageBytes = 34 * 1024;      // every stage starts 1024-byte aligned
-constexpr int kRedOffset = kStreamStages * kStageBytes;  // [8 warps][16 tokens][16 rows] fp32
-constexpr int kBarOffset = kRedOffset + kStreamConsumers * 16 * kStreamRows * 4;
+constexpr int kStV = kStMask + 2048;         // the step's 1024 col-axis scales
+constexpr int kStageBytes = 36 * 1024;      // every stage starts 1024-byte aligned
+constexpr int kRedOffset = 0;               // [8 warps][16 tokens][16 rows] fp32, over the ring once it has drained
+constexpr int kBarOffset = kStreamStages * kStageBytes;
+static_assert(kStreamConsumers * 16 * kStreamRows * 4 <= kStageBytes, "the reduction buffer reuses stage 0");
 constexpr int kStreamSmem = kBarOffset + 256 + 1024 /* alignment slack */;
 
 struct StreamArgs {
@@ -289,9 +291,9 @@ __device__ __forceinline__ uint4 ldg_cached(const void *p) {
     return r;
 }
 
-// x fragments of one 64-column block: [c] = piece t + 4c; a = token g, b = token g + 8, v = scales (col axis)
+// x fragments of one 64-column block: [c] = piece t + 4c; a = token g, b = token g + 8
 struct XFrag {
-    uint4 a[2], b[2], v[2];
+    uint4 a[2], b[2];
 };
 
 template <bool COL, bool M16>
@@ -303,7 +305,6 @@ __device__ __forceinline__ void load_xfrag(XFrag &f, const StreamArgs &a, int k0
         f.b[c] = make_uint4(0, 0, 0, 0);
         if (g < a.M) f.a[c] = ldg_cached(a.x + static_cast<size_t>(g) * a.ldx + k);
         if (M16 && g + 8 < a.M) f.b[c] = ldg_cached(a.x + static_cast<size_t>(g + 8) * a.ldx + k);
-        if (COL) f.v[c] = ldg_cached(a.v + k);
     }
 }
 
@@ -345,10 +346,12 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         !(ok = mbar_wait(empty + st, ((gs / kStreamStages) & 1) ^ 1, abort_flag, a.status, 11)))
                         break;
                     unsigned char *base = smem + st * kStageBytes;
-                    mbar_arrive_expect_tx(full + st, kTxBytes);
+                    const uint32_t v_bytes = kCol ? static_cast<uint32_t>(min(kStreamK, a.d_in - s * kStreamK) * 2) : 0u;
+                    mbar_arrive_expect_tx(full + st, kTxBytes + v_bytes);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) tma_load_3d(&map_w, full + st, base + kStW + q * 8192, 0, s * 16 + 4 * q, row0);
                     if (HAS_DELTA) tma_load_2d(&map_m, full + st, base + kStMask, s * 32, row0);
+                    if (kCol) bulk_load_1d(base + kStV, a.v + static_cast<size_t>(s) * kStreamK, v_bytes, full + st);
                 }
             }
         }
@@ -410,14 +413,17 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         const uint32_t in_row = static_cast<uint32_t>(bi * 128) +
                                                 ((static_cast<uint32_t>(t + 4 * c) ^ static_cast<uint32_t>(((g & 1) << 2) | bi)) << 4);
                         const uint4 xa = cur.a[c], xb = cur.b[c];
-                        // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis)
+                        // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis),
+                        // read from the stage (all lanes with the same t read the same 16 bytes: a broadcast)
+                        uint4 vv = make_uint4(0, 0, 0, 0);
+                        if (kCol) vv = *reinterpret_cast<const uint4 *>(smem + st * kStageBytes + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
                         uint32_t mg[2][4];
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            mg[j][0] = kCol ? cur.v[c].x : mag[j];
-                            mg[j][1] = kCol ? cur.v[c].y : mag[j];
-                            mg[j][2] = kCol ? cur.v[c].z : mag[j];
-                            mg[j][3] = kCol ? cur.v[c].w : mag[j];
+                            mg[j][0] = kCol ? vv.x : mag[j];
+                            mg[j][1] = kCol ? vv.y : mag[j];
+                            mg[j][2] = kCol ? vv.z : mag[j];
+                            mg[j][3] = kCol ? vv.w : mag[j];
                         }
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
