@@ -384,6 +384,31 @@ def test_multivariant_prefill_sized(api, d_out, d_in, n_var, m):
         assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
 
 
+@pytest.mark.parametrize("mixed_axes", [False, True])
+def test_multivariant_7b_shape_16_variants(api, mixed_axes):
+    # the multi-variant serving batch at full size on one 7B linear: 16 variants over one base, 64 decode rows
+    # (own id each) followed by 4 x 512 prefill rows; oracle on a fixed sample of rows
+    d_out = d_in = 4096
+    n_var = 16
+    w_b = synth.gen_base(d_out, d_in, 31)
+    masks, vs, axes = make_variants(w_b, n_var, 31, mixed_axes=mixed_axes, axis=ROW)
+    d_args = (dev(w_b), dev(masks), dev(vs))
+    for m, ids in ((64, synth.gen_ids(64, n_var, 33)), (2112, synth.gen_ids(2112, n_var, 34)),
+                   (2112, synth.gen_ids_per_sequence(64, 4, 512, n_var, 35))):
+        x = synth.gen_x(m, d_in, 32 + m)
+        y = api.pd_linear_multivariant(dev(x), dev(ids), d_args[0], d_args[1], d_args[2], axes)
+        torch.cuda.synchronize()
+        assert api.pd_device_status() == 0
+        rows = np.arange(m) if m <= 64 else synth.sample_rows(m, n_random=24)
+        ref, bad = orc.linear_multivariant(np.ascontiguousarray(x[rows]), np.ascontiguousarray(ids[rows]), w_b, masks, vs, axes)
+        assert bad == 0
+        yh = host(y).astype(np.float64)
+        assert np.isfinite(yh).all()
+        assert rel_err(yh[rows], ref) <= TOL
+        for i, r in enumerate(rows):  # row by row: no row may borrow another variant's delta
+            assert np.max(np.abs(yh[r] - ref[i])) / np.max(np.abs(ref[i])) <= 2 * TOL
+
+
 def test_multivariant_bad_id_is_latched(api):
     w_b = synth.gen_base(128, 128, 14)
     masks, vs, axes = make_variants(w_b, 2, 14)
