@@ -238,39 +238,41 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming decode kernel: weights brought in by TMA, one CTA per 16 output rows, two CTAs per SM.
+// Streaming decode kernel: weights brought in by TMA, one CTA per R output rows, two or three CTAs per SM.
 //
-// A CTA owns 16 rows for the whole of d_in, so its result needs no other CTA: no partial sums in
-// global memory, no tickets, no fences.  It walks d_in in steps of 1024 columns: 2 KB of contiguous
-// W_b per row and step (long row segments are what HBM delivers fastest: on B200 a pure TMA stream
-// of [16 rows x 2 KB] steps, three in flight per CTA, measured 6.1-7.1 TB/s on the 7B shapes,
-// against 4.4-5.4 TB/s for 512-byte segments).  A step is four TMA boxes of {64 columns, 4 blocks,
-// 16 rows} (128-byte swizzle; rows of 512 bytes keep the fragment reads conflict free) plus one box
-// of mask words: 34 KB, three steps in flight per CTA.
+// A CTA owns R rows (16; 32 compiles but measured slower) for the whole of d_in, so its result needs no other CTA: no partial
+// sums in global memory, no tickets, no fences.  It walks d_in in steps of 16384/R columns: 2 KB
+// (R = 16) or 1 KB (R = 32) of contiguous W_b per row and step (long row segments are what HBM
+// delivers fastest: on B200 a pure TMA stream of [16 rows x 2 KB] steps, three in flight per CTA,
+// measured 6.1-7.1 TB/s on the 7B shapes, against 4.4-5.4 TB/s for 512-byte segments).  A step is
+// 32 KB of W_b in boxes of {64 columns, 4 blocks, R rows} (128-byte swizzle; rows of 512 bytes keep
+// the fragment reads conflict free), one box of mask words and, for the col axis, a bulk copy of the
+// step's scales: 34-36 KB, two or three steps in flight per CTA (two when the grid is large enough
+// for three CTAs per SM).
 //
-// Eight consumer warps share every step: warp w takes the 64-column blocks 2w and 2w+1 and both n8
-// tiles.  W_b and mask come from shared memory; the x fragments (and v for the col axis) are read
-// straight from global memory -- x is small and L2-resident, and keeping it out of shared memory
-// leaves the ring to the weights.  The delta term enters the same accumulator as x . (+-s) with
-// s = v[row] (row axis) or s = v[k] (col axis): exact fp16 products summed in fp32 either way.
-// The eight warps' partial sums are added in warp order through shared memory.
+// The mask box is fetched through a map that sees the words as {4 words, rows, groups of 128
+// columns}: in shared memory the 16 bytes of one row and group sit next to those of the next row,
+// so the eight rows a warp reads at once fall into different banks.
 //
-// Programmatic dependent launch: W_b and mask do not depend on the previous kernel in the stream,
+// Eight consumer warps share every step: each takes one or two 64-column blocks and all R rows.
+// W_b, mask and the col-axis scales come from shared memory; the x fragments are read straight from
+// global memory -- x is small and L2-resident, and keeping it out of shared memory leaves the ring
+// to the weights.  The delta term enters the same accumulator as
+// x . (+-s) with s = v[row] (row axis) or s = v[k] (col axis): exact fp16 products summed in fp32
+// either way.  The eight warps' partial sums are added in warp order through shared memory.
+//
+// Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the stream,
 // so the producer starts loading at once; the consumers wait for the previous kernel
-// (griddepcontrol.wait) before they touch x, v or y.
-constexpr int kStreamRows = 16;
-constexpr int kStreamK = 1024;
-constexpr int kStreamStages = 3;
+// (griddepcontrol.wait) before they touch x or y.
 constexpr int kStreamConsumers = 8;
 constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
-constexpr int kStW = 0;                     // 4 boxes of [16 rows][4 blocks][128 B], swizzled (8 KB each)
-constexpr int kStMask = 32768;              // [16 rows][32 words]
-constexpr int kStV = kStMask + 2048;         // the step's 1024 col-axis scales
+constexpr int kStW = 0;                     // boxes of [R rows][4 blocks][128 B], swizzled: 32 KB
+constexpr int kStMask = 32768;              // [groups of 128 columns][R rows][4 words]: 2 KB
+constexpr int kStV = kStMask + 2048;        // the step's col-axis scales: up to 2 KB
 constexpr int kStageBytes = 36 * 1024;      // every stage starts 1024-byte aligned
-constexpr int kRedOffset = 0;               // [8 warps][16 tokens][16 rows] fp32, over the ring once it has drained
-constexpr int kBarOffset = kStreamStages * kStageBytes;
-static_assert(kStreamConsumers * 16 * kStreamRows * 4 <= kStageBytes, "the reduction buffer reuses stage 0");
-constexpr int kStreamSmem = kBarOffset + 256 + 1024 /* alignment slack */;
+constexpr int kRedOffset = 0;               // [8 warps][16 tokens][R rows] fp32, over the ring once it has drained
+static_assert(kStreamConsumers * 16 * 32 * 4 <= kStageBytes, "the reduction buffer reuses stage 0");
+constexpr int stream_smem_bytes(int stages) { return stages * kStageBytes + 256 + 1024 /* alignment slack */; }
 
 struct StreamArgs {
     const __half *x;
@@ -278,7 +280,7 @@ struct StreamArgs {
     __half *y;
     int64_t ldx, ldy;
     int M, d_out, d_in;
-    int n_k;      // steps of 1024 columns (the last one may be partly past d_in)
+    int n_k;      // steps of 16384/R columns (the last one may be partly past d_in)
     uint32_t *status;
 };
 
@@ -308,19 +310,24 @@ __device__ __forceinline__ void load_xfrag(XFrag &f, const StreamArgs &a, int k0
     }
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16>
-__global__ void __maxnreg__(96)
+template <int AXIS, bool HAS_DELTA, bool M16, int R, int STAGES>
+__global__ void __maxnreg__(STAGES == 2 ? 72 : 96)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float *red = reinterpret_cast<float *>(smem + kRedOffset);
-    uint64_t *full = reinterpret_cast<uint64_t *>(smem + kBarOffset);
+    constexpr int kStreamStages = STAGES;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * kStageBytes);
     uint64_t *empty = full + kStreamStages;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + kStreamStages);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr bool kCol = HAS_DELTA && AXIS == PD_AXIS_COL;
     constexpr uint32_t kTxBytes = 32768u + (HAS_DELTA ? 2048u : 0u);
+    constexpr int kStep = 16384 / R;           // columns per step
+    constexpr int kItems = kStep / 64 / kStreamConsumers;  // 64-column blocks per warp and step
+    constexpr int kTiles = R / 8;              // n8 tiles of output rows
+    static_assert(R == 16 || R == 32, "rows per CTA");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) {
@@ -339,153 +346,144 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             uint32_t gs = 0;           // steps issued so far
             bool ok = true;
             {
-                const int row0 = blockIdx.x * kStreamRows;
+                const int row0 = blockIdx.x * R;
                 for (int s = 0; s < a.n_k; ++s, ++gs) {
                     const int st = gs % kStreamStages;
                     if (gs >= kStreamStages &&
                         !(ok = mbar_wait(empty + st, ((gs / kStreamStages) & 1) ^ 1, abort_flag, a.status, 11)))
                         break;
                     unsigned char *base = smem + st * kStageBytes;
-                    const uint32_t v_bytes = kCol ? static_cast<uint32_t>(min(kStreamK, a.d_in - s * kStreamK) * 2) : 0u;
+                    const uint32_t v_bytes = kCol ? static_cast<uint32_t>(min(kStep, a.d_in - s * kStep) * 2) : 0u;
                     mbar_arrive_expect_tx(full + st, kTxBytes + v_bytes);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) tma_load_3d(&map_w, full + st, base + kStW + q * 8192, 0, s * 16 + 4 * q, row0);
-                    if (HAS_DELTA) tma_load_2d(&map_m, full + st, base + kStMask, s * 32, row0);
-                    if (kCol) bulk_load_1d(base + kStV, a.v + static_cast<size_t>(s) * kStreamK, v_bytes, full + st);
+                    for (int q = 0; q < kStep / 256; ++q)
+                        tma_load_3d(&map_w, full + st, base + kStW + q * (R * 512), 0, s * (kStep / 64) + 4 * q, row0);
+                    if (HAS_DELTA) tma_load_3d(&map_m, full + st, base + kStMask, 0, row0, s * (kStep / 128));
+                    if (kCol) bulk_load_1d(base + kStV, a.v + static_cast<size_t>(s) * kStep, v_bytes, full + st);
                 }
             }
         }
     } else {
         // ------------------------------------------------ consumers
         const int g = lane >> 2, t = lane & 3;
-        const uint32_t sel_t = static_cast<uint32_t>(t | ((4 + t) << 4));
+        const uint32_t byte_t = static_cast<uint32_t>(t) | 0x4440u;  // prmt: byte t of the first operand, zeros above
         grid_dependency_wait();  // x may be the previous kernel's output
-        const int n_items = 2 * a.n_k;
-        auto item_k0 = [&](int it) { return (it >> 1) * kStreamK + (2 * warp + (it & 1)) * 64; };
+        const int n_items = kItems * a.n_k;
+        auto item_k0 = [&](int it) { return (it / kItems) * kStep + (kItems * warp + (it % kItems)) * 64; };
         uint32_t gs = 0;  // steps consumed so far
         bool ok = true;
-        do {  // one tile per CTA
-            const int row0 = blockIdx.x * kStreamRows;
-            float acc[2][4];
+        const int row0 = blockIdx.x * R;
+        float acc[kTiles][4];
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
+        for (int j = 0; j < kTiles; ++j)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
-            uint32_t mag[2];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
+            for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
+        uint32_t mag[kTiles];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                mag[j] = 0x3C003C00u;
-                if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
-                    const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
-                    mag[j] = h | (h << 16);
-                }
+        for (int j = 0; j < kTiles; ++j) {
+            mag[j] = 0x3C003C00u;
+            if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
+                const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
+                mag[j] = h | (h << 16);
             }
-            // items: (step s, block bb of this warp), k0 = s*1024 + (2*warp + bb)*64; x fragments one item ahead
-            // (two ahead for up to 8 tokens, where the registers allow it: the loads come from L2, ~1 us away under load)
-            constexpr int kAhead = M16 ? 1 : 2;
-            XFrag cur, nxt, nxt2;
-            if (item_k0(0) < a.d_in) load_xfrag<kCol, M16>(cur, a, item_k0(0), g, t);
-            if (kAhead == 2 && 1 < n_items && item_k0(1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(1), g, t);
-            for (int it = 0; it < n_items && ok; ++it) {
-                const int bb = it & 1, st = gs % kStreamStages;
-                const int k0 = item_k0(it);
-                if (kAhead == 1) {
-                    if (it + 1 < n_items && item_k0(it + 1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(it + 1), g, t);
-                } else {
-                    if (it + 2 < n_items && item_k0(it + 2) < a.d_in) load_xfrag<kCol, M16>(nxt2, a, item_k0(it + 2), g, t);
+        }
+        // items: (step s, block bb of this warp), k0 = s*kStep + (kItems*warp + bb)*64; x fragments one item ahead
+        // (two ahead for up to 8 tokens, where the registers allow it: the loads come from L2, ~1 us away under load)
+        constexpr int kAhead = M16 ? 1 : 2;
+        XFrag cur, nxt, nxt2;
+        if (item_k0(0) < a.d_in) load_xfrag<kCol, M16>(cur, a, item_k0(0), g, t);
+        if (kAhead == 2 && 1 < n_items && item_k0(1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(1), g, t);
+        for (int it = 0; it < n_items && ok; ++it) {
+            const int bb = it % kItems, st = gs % kStreamStages;
+            const int k0 = item_k0(it);
+            if (kAhead == 1) {
+                if (it + 1 < n_items && item_k0(it + 1) < a.d_in) load_xfrag<kCol, M16>(nxt, a, item_k0(it + 1), g, t);
+            } else {
+                if (it + 2 < n_items && item_k0(it + 2) < a.d_in) load_xfrag<kCol, M16>(nxt2, a, item_k0(it + 2), g, t);
+            }
+            if (bb == 0 && !(ok = mbar_wait(full + st, (gs / kStreamStages) & 1, abort_flag, a.status, 12))) break;
+            if (k0 < a.d_in) {  // else past the end of d_in: W was zero-filled there and x must not be read
+                const int blk = kItems * warp + bb;                   // block inside the step
+                const unsigned char *stage = smem + st * kStageBytes;
+                const unsigned char *box = stage + kStW + (blk >> 2) * (R * 512);
+                const int bi = blk & 3;                               // block inside its box
+                uint2 mw[kTiles];                                     // the block's 64 sign bits of rows 8j + g
+                if (HAS_DELTA) {
+#pragma unroll
+                    for (int j = 0; j < kTiles; ++j)
+                        mw[j] = *reinterpret_cast<const uint2 *>(stage + kStMask + (blk >> 1) * (R * 16) + (8 * j + g) * 16 + (blk & 1) * 8);
                 }
-                if (bb == 0 && !(ok = mbar_wait(full + st, (gs / kStreamStages) & 1, abort_flag, a.status, 12))) break;
-                if (k0 < a.d_in) {  // else past the end of d_in: W was zero-filled there and x must not be read
-                    const int blk = 2 * warp + bb;                       // block inside the step
-                    const unsigned char *box = smem + st * kStageBytes + kStW + (blk >> 2) * 8192;
-                    const int bi = blk & 3;                               // block inside its box
-                    uint32_t my[2];                                       // per tile: byte c = sign bits of piece t + 4c
-                    if (HAS_DELTA) {
 #pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const uint2 m = *reinterpret_cast<const uint2 *>(smem + st * kStageBytes + kStMask + (8 * j + g) * 128 + blk * 8);
-                            my[j] = prmt(m.x, m.y, sel_t);
-                        }
-                    }
+                for (int c = 0; c < 2; ++c) {
+                    // byte offset inside a 512-byte row of the box, swizzled: piece index ^ (bits 7..9 of the offset)
+                    const uint32_t in_row = static_cast<uint32_t>(bi * 128) +
+                                            ((static_cast<uint32_t>(t + 4 * c) ^ static_cast<uint32_t>(((g & 1) << 2) | bi)) << 4);
+                    const uint4 xa = cur.a[c], xb = cur.b[c];
+                    // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis),
+                    // read from the stage (all lanes with the same t read the same 16 bytes: a broadcast)
+                    uint4 vv = make_uint4(0, 0, 0, 0);
+                    if (kCol) vv = *reinterpret_cast<const uint4 *>(stage + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        // byte offset inside a 512-byte row of the box, swizzled: piece index ^ (bits 7..9 of the offset)
-                        const uint32_t in_row = static_cast<uint32_t>(bi * 128) +
-                                                ((static_cast<uint32_t>(t + 4 * c) ^ static_cast<uint32_t>(((g & 1) << 2) | bi)) << 4);
-                        const uint4 xa = cur.a[c], xb = cur.b[c];
-                        // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis),
-                        // read from the stage (all lanes with the same t read the same 16 bytes: a broadcast)
-                        uint4 vv = make_uint4(0, 0, 0, 0);
-                        if (kCol) vv = *reinterpret_cast<const uint4 *>(smem + st * kStageBytes + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
-                        uint32_t mg[2][4];
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            mg[j][0] = kCol ? vv.x : mag[j];
-                            mg[j][1] = kCol ? vv.y : mag[j];
-                            mg[j][2] = kCol ? vv.z : mag[j];
-                            mg[j][3] = kCol ? vv.w : mag[j];
-                        }
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
-                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
-                            if (HAS_DELTA) {
-                                // pair r = halves 2r, 2r+1 of the piece: bit 2r of byte c -> bit 15, bit 2r+1 -> bit 31;
-                                // a clear bit (B = -1) flips the sign of the magnitude
-                                const uint32_t sel = static_cast<uint32_t>(((c | 8) << 4) | (((4 + c) | 8) << 12));
-                                uint32_t pm[4];
-#pragma unroll
-                                for (int r = 0; r < 4; ++r)
-                                    pm[r] = lop3_andn_xor(prmt(my[j] << (7 - 2 * r), my[j] << (6 - 2 * r), sel), 0x80008000u, mg[j][r]);
-                                mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm[0], pm[1]);
-                                mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm[2], pm[3]);
-                            }
+                    for (int j = 0; j < kTiles; ++j) {
+                        const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
+                        mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                        mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                        if (HAS_DELTA) {
+                            // the piece's 8 sign bits are byte t of word c.  b * 0x8001 puts bit i at i and i + 15,
+                            // so a left shift by 15 - 2r brings bit 2r to bit 15 and bit 2r + 1 to bit 31: the signs
+                            // of halves 2r, 2r + 1.  A clear bit (B = -1) flips the sign of the magnitude.
+                            const uint32_t sp = prmt(c ? mw[j].y : mw[j].x, 0u, byte_t) * 0x8001u;
+                            const uint32_t pm0 = lop3_andn_xor(sp << 15, 0x80008000u, kCol ? vv.x : mag[j]);
+                            const uint32_t pm1 = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
+                            const uint32_t pm2 = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
+                            const uint32_t pm3 = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
+                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm0, pm1);
+                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm2, pm3);
                         }
                     }
                 }
-                if (bb == 1) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(empty + st);
-                    ++gs;
-                }
-                cur = nxt;
-                if (kAhead == 2) nxt = nxt2;
             }
+            if (bb == kItems - 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + st);
+                ++gs;
+            }
+            cur = nxt;
+            if (kAhead == 2) nxt = nxt2;
+        }
 
-            // ---- add the eight warps' partial sums in warp order.  The first barrier ORs "a wait ran out"
-            // over the consumers, so that all of them leave together.
-            uint32_t gave_up;
-            asm volatile(
-                "{\n"
-                ".reg .pred p, q;\n"
-                "setp.ne.u32 q, %1, 0;\n"
-                "bar.red.or.pred p, 1, %2, q;\n"
-                "selp.u32 %0, 1, 0, p;\n"
-                "}\n"
-                : "=r"(gave_up)
-                : "r"(static_cast<uint32_t>(!ok || *abort_flag)), "n"(kStreamConsumers * 32)
-                : "memory");
-            if (gave_up) break;
-            float *mine = red + warp * 16 * kStreamRows;  // [16 tokens][16 rows]
+        // ---- add the eight warps' partial sums in warp order.  The first barrier ORs "a wait ran out"
+        // over the consumers, so that all of them leave together.
+        uint32_t gave_up;
+        asm volatile(
+            "{\n"
+            ".reg .pred p, q;\n"
+            "setp.ne.u32 q, %1, 0;\n"
+            "bar.red.or.pred p, 1, %2, q;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(gave_up)
+            : "r"(static_cast<uint32_t>(!ok || *abort_flag)), "n"(kStreamConsumers * 32)
+            : "memory");
+        if (!gave_up) {
+            float *mine = red + warp * 16 * R;  // [16 tokens][R rows]
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
+            for (int j = 0; j < kTiles; ++j)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int ol = 8 * j + 2 * t + e;
-                    mine[g * kStreamRows + ol] = acc[j][e];
-                    mine[(g + 8) * kStreamRows + ol] = acc[j][2 + e];
+                    mine[g * R + ol] = acc[j][e];
+                    mine[(g + 8) * R + ol] = acc[j][2 + e];
                 }
             asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
-            {
-                const int idx = threadIdx.x;  // 256 consumer threads = 16 tokens x 16 rows
-                const int tok = idx >> 4, ol = idx & 15;
+            for (int idx = threadIdx.x; idx < 16 * R; idx += kStreamConsumers * 32) {  // (token, row) pairs
+                const int tok = idx / R, ol = idx % R;
                 float sum = 0.f;
 #pragma unroll
-                for (int w = 0; w < kStreamConsumers; ++w) sum += red[(w * 16 + tok) * kStreamRows + ol];
+                for (int w = 0; w < kStreamConsumers; ++w) sum += red[(w * 16 + tok) * R + ol];
                 if (tok < a.M && row0 + ol < a.d_out) a.y[static_cast<size_t>(tok) * a.ldy + row0 + ol] = __float2half_rn(sum);
             }
-        } while (false);
+        }
     }
 }
 
@@ -575,10 +573,11 @@ pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) 
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, args));
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16>
+template <int AXIS, bool HAS_DELTA, bool M16, int R, int STAGES>
 pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, const StreamArgs &args, int grid,
                                 cudaStream_t stream) {
-    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16>;
+    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16, R, STAGES>;
+    constexpr int kStreamSmem = stream_smem_bytes(STAGES);
     static bool configured = false;  // per instantiation
     if (!configured) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem) != cudaSuccess)
@@ -600,16 +599,16 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, co
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mm, args));
 }
 
-pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
-                        int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                        cudaStream_t stream) {
+template <int R, int STAGES>
+pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
+                             int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                             cudaStream_t stream) {
+    constexpr int step = 16384 / R;
     const bool m16 = M > 8, delta = mask != nullptr;
     CUtensorMap mw, mm;
-    if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, kStreamRows)) return PD_ERR_CUDA;
+    if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, R)) return PD_ERR_CUDA;
     mm = mw;
-    if (delta && !make_map_2d(&mm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, mask, d_out, d_in / 32, d_in / 8, 32, kStreamRows,
-                              CU_TENSOR_MAP_SWIZZLE_NONE))
-        return PD_ERR_CUDA;
+    if (delta && !make_map_mask_groups(&mm, mask, d_out, d_in, R, step / 128)) return PD_ERR_CUDA;
     StreamArgs a;
     a.x = x;
     a.v = v;
@@ -619,12 +618,12 @@ pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, 
     a.M = M;
     a.d_out = static_cast<int>(d_out);
     a.d_in = static_cast<int>(d_in);
-    a.n_k = static_cast<int>((d_in + kStreamK - 1) / kStreamK);
+    a.n_k = static_cast<int>((d_in + step - 1) / step);
     a.status = status;
-    // one CTA per tile of 16 rows: a persistent grid walking several tiles measured slower on the 7B
+    // one CTA per tile of R rows: a persistent grid walking several tiles measured slower on the 7B
     // shapes (fewer rings in flight, more registers)
-    const int grid = static_cast<int>((d_out + kStreamRows - 1) / kStreamRows);
-#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W>(mw, mm, a, grid, stream)
+    const int grid = static_cast<int>((d_out + R - 1) / R);
+#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W, R, STAGES>(mw, mm, a, grid, stream)
     if (!delta) {
         if (m16) PD_STREAM_CASE(PD_AXIS_ROW, false, true);
         PD_STREAM_CASE(PD_AXIS_ROW, false, false);
@@ -636,6 +635,23 @@ pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, 
     if (m16) PD_STREAM_CASE(PD_AXIS_COL, true, true);
     PD_STREAM_CASE(PD_AXIS_COL, true, false);
 #undef PD_STREAM_CASE
+}
+
+pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
+                        int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                        cudaStream_t stream) {
+    // Ring depth.  A two-step ring lets three CTAs share an SM: the same bytes in flight, but a CTA that is
+    // finishing (last step, reduction, store) overlaps two that stream.  It needs a grid that fills three CTAs
+    // per SM (smaller grids need the third step per CTA to keep enough in flight) and whose last wave is not
+    // much emptier than with two CTAs per SM.  Tiles of 32 rows (half the x traffic) measured slower on every
+    // 7B shape: too few consumer warps per SM when the grid is small.
+    static const int forced = env_int("PD_GEMV_STAGES", 0);
+    const double tiles = static_cast<double>((d_out + 15) / 16);
+    const double w2 = tiles / (3.0 * sm_count()), w3 = tiles / (2.0 * sm_count());
+    const bool two = w2 >= 1.0 && w2 / ceil(w2) >= w3 / ceil(w3) - 0.1;
+    const int stages = forced ? forced : (two ? 2 : 3);
+    if (stages == 2) return launch_stream_rows<16, 2>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    return launch_stream_rows<16, 3>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
 }
 
 }  // namespace

@@ -161,6 +161,22 @@ inline bool make_map_blocked_f16(CUtensorMap *map, const void *base, int64_t row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Packed mask [rows, cols/32 words] (cols a multiple of 128) seen as {4 words, rows, cols/128 groups}: one box of
+// {4, box_rows, box_groups} lands in shared memory as [group][row][4 words], i.e. the 16 bytes of consecutive
+// rows are adjacent.  Groups past the end read as zeros.
+inline bool make_map_mask_groups(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int box_rows,
+                                 int box_groups) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {4, static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(cols / 128)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(cols / 8), 16};
+    const cuuint32_t box[3] = {4, static_cast<cuuint32_t>(box_rows), static_cast<cuuint32_t>(box_groups)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline int sm_count() {
     static int n = [] {
         int dev = 0, v = 0;
