@@ -238,41 +238,47 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Streaming decode kernel: weights brought in by TMA, one CTA per R output rows, two or three CTAs per SM.
+// Streaming decode kernel: weights brought in by TMA, one CTA per 16 output rows, two or three CTAs per SM.
 //
-// A CTA owns R rows (16; 32 compiles but measured slower) for the whole of d_in, so its result needs no other CTA: no partial
-// sums in global memory, no tickets, no fences.  It walks d_in in steps of 16384/R columns: 2 KB
-// (R = 16) or 1 KB (R = 32) of contiguous W_b per row and step (long row segments are what HBM
-// delivers fastest: on B200 a pure TMA stream of [16 rows x 2 KB] steps, three in flight per CTA,
-// measured 6.1-7.1 TB/s on the 7B shapes, against 4.4-5.4 TB/s for 512-byte segments).  A step is
-// 32 KB of W_b in boxes of {64 columns, 4 blocks, R rows} (128-byte swizzle; rows of 512 bytes keep
-// the fragment reads conflict free), one box of mask words and, for the col axis, a bulk copy of the
-// step's scales: 34-36 KB, two or three steps in flight per CTA (two when the grid is large enough
-// for three CTAs per SM).
+// A CTA owns 16 rows for the whole of d_in, so its result needs no other CTA: no partial sums in
+// global memory, no tickets, no fences.  It walks d_in in steps of 512 columns: 1 KB of contiguous
+// W_b per row and step (HBM wants long row segments: on B200 a pure TMA stream of [16 rows x 2 KB]
+// steps measured 6.1-7.1 TB/s on the 7B shapes against 4.4-5.4 TB/s for 512-byte segments; 1 KB
+// steps run as fast as 2 KB ones here and halve what the consumers still have to do once the last
+// bytes have landed).  A step is 16 KB of W_b in two boxes of {64 columns, 4 blocks, 16 rows}
+// (128-byte swizzle; rows of 512 bytes keep the fragment reads conflict free), one box of mask
+// words and, for the col axis, a bulk copy of the step's scales: 17-18 KB.  A CTA keeps six steps
+// in flight (two CTAs per SM), or four (three CTAs per SM) when the grid is large enough.
 //
 // The mask box is fetched through a map that sees the words as {4 words, rows, groups of 128
 // columns}: in shared memory the 16 bytes of one row and group sit next to those of the next row,
 // so the eight rows a warp reads at once fall into different banks.
 //
-// Eight consumer warps share every step: each takes one or two 64-column blocks and all R rows.
-// W_b, mask and the col-axis scales come from shared memory; the x fragments are read straight from
-// global memory -- x is small and L2-resident, and keeping it out of shared memory leaves the ring
-// to the weights.  The delta term enters the same accumulator as
-// x . (+-s) with s = v[row] (row axis) or s = v[k] (col axis): exact fp16 products summed in fp32
-// either way.  The eight warps' partial sums are added in warp order through shared memory.
+// Eight consumer warps share every step: each takes one 64-column block and all 16 rows.  W_b, mask
+// and the col-axis scales come from shared memory; the x fragments are read straight from global
+// memory -- x is small and L2-resident, and keeping it out of shared memory leaves the ring to the
+// weights.  The delta term enters the same accumulator as x . (+-s) with s = v[row] (row axis) or
+// s = v[k] (col axis): exact fp16 products summed in fp32 either way.  The eight warps' partial
+// sums are added in warp order through shared memory.
 //
 // Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the stream,
 // so the producer starts loading at once; the consumers wait for the previous kernel
 // (griddepcontrol.wait) before they touch x or y.
 constexpr int kStreamConsumers = 8;
 constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
-constexpr int kStW = 0;                     // boxes of [R rows][4 blocks][128 B], swizzled: 32 KB
-constexpr int kStMask = 32768;              // [groups of 128 columns][R rows][4 words]: 2 KB
-constexpr int kStV = kStMask + 2048;        // the step's col-axis scales: up to 2 KB
-constexpr int kStageBytes = 36 * 1024;      // every stage starts 1024-byte aligned
+constexpr int kStreamRows = 16;             // output rows per CTA
+// one stage of KS columns: W_b boxes of [16 rows][4 blocks][128 B], swizzled; mask as [groups of 128 columns]
+// [rows][4 words]; the step's col-axis scales.  36 bytes per column: every stage starts 1024-byte aligned.
+constexpr int kStW = 0;
+__host__ __device__ constexpr int stage_mask_offset(int ks) { return kStreamRows * ks * 2; }
+__host__ __device__ constexpr int stage_v_offset(int ks) { return stage_mask_offset(ks) + kStreamRows * ks / 8; }
+__host__ __device__ constexpr int stage_bytes(int ks) { return stage_v_offset(ks) + ks * 2; }
 constexpr int kRedOffset = 0;               // [8 warps][16 tokens][R rows] fp32, over the ring once it has drained
-static_assert(kStreamConsumers * 16 * 32 * 4 <= kStageBytes, "the reduction buffer reuses stage 0");
-constexpr int stream_smem_bytes(int stages) { return stages * kStageBytes + 256 + 1024 /* alignment slack */; }
+static_assert(kStreamConsumers * 16 * kStreamRows * 4 <= stage_bytes(512), "the reduction buffer reuses stage 0");
+static_assert(stage_bytes(512) % 1024 == 0 && stage_bytes(1024) % 1024 == 0, "stage alignment");
+constexpr int stream_smem_bytes(int ks, int stages) { return stages * stage_bytes(ks) + 256 + 1024 /* alignment slack */; }
+// three CTAs per SM when a CTA's ring is at most 72 KB (and the registers are capped accordingly)
+__host__ __device__ constexpr bool stream_three_per_sm(int ks, int stages) { return stages * stage_bytes(ks) <= 72 * 1024; }
 
 struct StreamArgs {
     const __half *x;
@@ -280,7 +286,7 @@ struct StreamArgs {
     __half *y;
     int64_t ldx, ldy;
     int M, d_out, d_in;
-    int n_k;      // steps of 16384/R columns (the last one may be partly past d_in)
+    int n_k;      // steps of KS columns (the last one may be partly past d_in)
     uint32_t *status;
 };
 
@@ -310,24 +316,26 @@ __device__ __forceinline__ void load_xfrag(XFrag &f, const StreamArgs &a, int k0
     }
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16, int R, int STAGES>
-__global__ void __maxnreg__(STAGES == 2 ? 72 : 96)
+template <int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
+__global__ void __maxnreg__(stream_three_per_sm(KS, STAGES) ? 72 : 96)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float *red = reinterpret_cast<float *>(smem + kRedOffset);
     constexpr int kStreamStages = STAGES;
+    constexpr int R = kStreamRows;
+    constexpr int kStageBytes = stage_bytes(KS), kStMask = stage_mask_offset(KS), kStV = stage_v_offset(KS);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + STAGES * kStageBytes);
     uint64_t *empty = full + kStreamStages;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(empty + kStreamStages);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr bool kCol = HAS_DELTA && AXIS == PD_AXIS_COL;
-    constexpr uint32_t kTxBytes = 32768u + (HAS_DELTA ? 2048u : 0u);
-    constexpr int kStep = 16384 / R;           // columns per step
+    constexpr uint32_t kTxBytes = static_cast<uint32_t>(kStreamRows) * (KS * 2u + (HAS_DELTA ? KS / 8u : 0u));
+    constexpr int kStep = KS;                  // columns per step
     constexpr int kItems = kStep / 64 / kStreamConsumers;  // 64-column blocks per warp and step
     constexpr int kTiles = R / 8;              // n8 tiles of output rows
-    static_assert(R == 16 || R == 32, "rows per CTA");
+    static_assert(KS == 512 || KS == 1024, "columns per step");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) {
@@ -573,11 +581,11 @@ pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) 
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, args));
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16, int R, int STAGES>
+template <int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
 pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, const StreamArgs &args, int grid,
                                 cudaStream_t stream) {
-    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16, R, STAGES>;
-    constexpr int kStreamSmem = stream_smem_bytes(STAGES);
+    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16, KS, STAGES>;
+    constexpr int kStreamSmem = stream_smem_bytes(KS, STAGES);
     static bool configured = false;  // per instantiation
     if (!configured) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem) != cudaSuccess)
@@ -599,11 +607,11 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, co
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mm, args));
 }
 
-template <int R, int STAGES>
+template <int KS, int STAGES>
 pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                              int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
                              cudaStream_t stream) {
-    constexpr int step = 16384 / R;
+    constexpr int step = KS, R = kStreamRows;
     const bool m16 = M > 8, delta = mask != nullptr;
     CUtensorMap mw, mm;
     if (!make_map_blocked_f16(&mw, w_b, d_out, d_in, d_in * 2, 4, R)) return PD_ERR_CUDA;
@@ -623,7 +631,7 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
     // one CTA per tile of R rows: a persistent grid walking several tiles measured slower on the 7B
     // shapes (fewer rings in flight, more registers)
     const int grid = static_cast<int>((d_out + R - 1) / R);
-#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W, R, STAGES>(mw, mm, a, grid, stream)
+#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W, KS, STAGES>(mw, mm, a, grid, stream)
     if (!delta) {
         if (m16) PD_STREAM_CASE(PD_AXIS_ROW, false, true);
         PD_STREAM_CASE(PD_AXIS_ROW, false, false);
@@ -640,18 +648,18 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
 pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                         int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
                         cudaStream_t stream) {
-    // Ring depth.  A two-step ring lets three CTAs share an SM: the same bytes in flight, but a CTA that is
-    // finishing (last step, reduction, store) overlaps two that stream.  It needs a grid that fills three CTAs
-    // per SM (smaller grids need the third step per CTA to keep enough in flight) and whose last wave is not
-    // much emptier than with two CTAs per SM.  Tiles of 32 rows (half the x traffic) measured slower on every
-    // 7B shape: too few consumer warps per SM when the grid is small.
-    static const int forced = env_int("PD_GEMV_STAGES", 0);
-    const double tiles = static_cast<double>((d_out + 15) / 16);
-    const double w2 = tiles / (3.0 * sm_count()), w3 = tiles / (2.0 * sm_count());
-    const bool two = w2 >= 1.0 && w2 / ceil(w2) >= w3 / ceil(w3) - 0.1;
-    const int stages = forced ? forced : (two ? 2 : 3);
-    if (stages == 2) return launch_stream_rows<16, 2>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
-    return launch_stream_rows<16, 3>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    // Ring depth.  A shorter ring (four steps, 72 KB) lets three CTAs share an SM: the same bytes in flight,
+    // but a CTA that is finishing (last step, reduction, store) overlaps two that stream.  It needs a grid that
+    // fills three CTAs per SM (smaller grids need six steps per CTA to keep enough in flight) and whose last
+    // wave is not much emptier than with two CTAs per SM.  Measured and dropped: tiles of 32 rows (half the x
+    // traffic, but too few consumer warps per SM on small grids) and tiles of 12-15 rows (fill every SM when
+    // d_out / 16 is just under a wave, but the consumers' work per CTA does not shrink with the tile).
+    static const int forced = env_int("PD_GEMV_CTAS_PER_SM", 0);  // 2 or 3; 0 = by the rule below
+    const double tiles = static_cast<double>((d_out + kStreamRows - 1) / kStreamRows);
+    const double w3 = tiles / (3.0 * sm_count()), w2 = tiles / (2.0 * sm_count());
+    const bool three = forced ? forced == 3 : (w3 >= 1.0 && w3 / ceil(w3) >= w2 / ceil(w2) - 0.1);
+    if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
 }
 
 }  // namespace
