@@ -25,6 +25,8 @@
 // warps take the even steps, four the odd ones.
 // Every wait is bounded; a wait that runs out latches PD_ERR_DEVICE_TIMEOUT and the CTA
 // drains and exits.
+#include <cstdlib>
+
 #include "pd_ptx.cuh"
 
 namespace pd {
@@ -467,6 +469,354 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     }
 }
 
+// ------------------------------------------------------------------ CTA-pair kernel (M >= 256, one variant)
+//
+// Two CTAs of a cluster (two SMs) work on one tile of 256 output rows x 256 tokens with
+// tcgen05.mma.cta_group::2: each CTA expands its own 128 rows of W_hat into its own tensor memory and
+// holds only HALF of the x tile (128 tokens) in shared memory; the tensor cores of both SMs read both
+// halves.  Per k step a CTA therefore moves 16 KB of x instead of 32 KB through shared memory, twice
+// (TMA fill, operand read): shared-memory bandwidth, which caps the one-CTA kernel at about two thirds
+// of the tensor peak, is no longer the limit.
+//
+// Rank 0 of the pair issues every MMA.  Barriers that gate it live in rank 0 only:
+//   ready[it % 8]   : 4 transform warps of each CTA (rank 1 arrives remotely) + rank 0's x producer, which also
+//                     announces the bytes of BOTH x halves; rank 1's TMA reports its bytes to rank 0's barrier
+//   acc_empty       : the 4 epilogue warps of each CTA
+// consumed[] and acc_full exist in both CTAs; one multicast tcgen05.commit arrives on both copies.
+// The W_b ring, its barriers and the transform are per CTA, as in the kernel above.
+struct PairLayout {
+    static constexpr int kStages = 6;             // x ring and W_b ring
+    static constexpr int kWBytes = BM * BK * 2;   // 16 KB
+    static constexpr int kXBytes = 128 * BK * 2;  // this CTA's half of the token tile: 16 KB
+    static constexpr int kXOffset = 0;
+    static constexpr int kWOffset = kStages * kXBytes;
+    static constexpr int kBarOffset = kWOffset + kStages * kWBytes;
+    static constexpr int kVOffset = kBarOffset + 512;
+    static constexpr int kOutOffset = kVOffset + kStages * kVSlotBytes;
+    static constexpr int kTotal = kOutOffset + 128 * 128 * 2 + 1024;
+    static_assert(kStages % 2 == 0 && kStages <= kASlots, "ring depth");
+    static_assert(kTotal <= 227 * 1024, "shared memory per CTA");
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `p` (a shared-memory object of this CTA) in the CTA of the given rank
+__device__ __forceinline__ uint32_t map_to_rank(const void *p, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// mbar_wait for a barrier that the other CTA of the pair arrives on
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                                  uint32_t where) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (true) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                latch_error(status, PD_ERR_DEVICE_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+}
+// x half of this CTA; the bytes are reported to the barrier at `bar_cluster_addr` (rank 0's)
+__device__ __forceinline__ void tma_load_2d_pair(const CUtensorMap *map, uint32_t bar_cluster_addr, void *dst, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_alloc_pair(uint32_t *dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at the same offset in both CTAs of the pair once the MMAs issued so far have completed
+__device__ __forceinline__ void tcgen05_commit_pair(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                     smem_u32(bar)),
+                 "h"(static_cast<unsigned short>(3))
+                 : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_f16_tmem_a_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                            uint32_t accumulate) {
+    const uint32_t z = 0;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z)
+        : "memory");
+}
+
+template <int AXIS, bool HAS_DELTA>
+__global__ void __launch_bounds__(kNumThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
+    using L = PairLayout;
+    constexpr int BN = 256;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
+    uint64_t *w_full = bars, *w_empty = bars + kMaxStages;
+    uint64_t *ready = bars + 2 * kMaxStages, *consumed = ready + kASlots;
+    uint64_t *acc_full = consumed + kASlots, *acc_empty = acc_full + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0 issues the MMAs
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int tiles_m2 = (a.tiles_m + 1) >> 1;        // tiles of 256 rows
+    const int n_tiles = tiles_m2 * a.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < L::kStages; ++s) {
+            mbar_init(w_full + s, 1);
+            mbar_init(w_empty + s, kXformWarps / 2);
+        }
+        for (int s = 0; s < kASlots; ++s) {
+            mbar_init(ready + s, 2 * (kXformWarps / 2) + 1);  // used in rank 0 only
+            mbar_init(consumed + s, 1);
+        }
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 2 * kEpiWarps);                   // used in rank 0 only
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < L::kStages * kVSlotBytes / 4) {
+        reinterpret_cast<uint32_t *>(smem + L::kVOffset)[threadIdx.x] = 0u;
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) tcgen05_alloc_pair(tmem_slot, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the other CTA's barriers are initialised before anything arrives on them
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // tile -> (256-row tile, token tile); this CTA's 128 rows and 128 tokens
+    auto tile_rows = [&](int tile) { return (tile / a.tiles_n) * 2 + static_cast<int>(rank); };      // W row tile of 128
+    auto tile_tok0 = [&](int tile) { return (tile % a.tiles_n) * BN; };
+
+    if (warp == 0 || warp == kNumWarps - 1) {
+        // ------------------------------------------------ TMA producers
+        if (lane == 0) {
+            const bool is_x = warp == 0;
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+                const int tm = tile_rows(tile), tok0 = tile_tok0(tile);
+                for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
+                    const int s = it % L::kStages;
+                    if (is_x) {
+                        if (it >= static_cast<uint32_t>(L::kStages)) {
+                            const uint32_t prev = it - L::kStages;
+                            if (!(ok = mbar_wait(consumed + prev % kASlots, (prev / kASlots) & 1, abort_flag, a.status, 1))) break;
+                        }
+                        uint64_t *rb = ready + it % kASlots;
+                        if (rank == 0) mbar_arrive_expect_tx(rb, 2 * L::kXBytes);  // both halves report here
+                        tma_load_2d_pair(&map_x, map_to_rank(rb, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
+                                         tok0 + 128 * static_cast<int>(rank));
+                    } else {
+                        const uint32_t parity = ((it / L::kStages) & 1) ^ 1;
+                        if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
+                        const uint32_t v_bytes = (HAS_DELTA && AXIS == PD_AXIS_COL) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
+                        mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
+                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, tm * BM);
+                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, a.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (rank 0 only): M = 256 over both CTAs, N = 256
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
+            for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
+                if (!(ok = mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, a.status, 2))) break;
+                tcgen05_fence_after();
+                for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
+                    const int s = it % L::kStages, sa = it % kASlots;
+                    if (!(ok = mbar_wait(ready + sa, (it / kASlots) & 1, abort_flag, a.status, 3))) break;
+                    tcgen05_fence_after();
+                    const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kXBytes);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tcgen05_mma_f16_tmem_a_pair(tmem_base, tmem_base + kACol0 + sa * 32 + kk * 8, make_smem_desc(x_addr + kk * 32),
+                                                    idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    tcgen05_commit_pair(consumed + sa);
+                }
+                if (ok) tcgen05_commit_pair(acc_full);
+            }
+        }
+    } else if (warp < 2 + kEpiWarps) {
+        // ------------------------------------------------ epilogue: this CTA's 128 rows of the accumulator, as in the kernel above
+        const int quarter = warp & 3;
+        const int et = threadIdx.x - 2 * 32;
+        unsigned char *stage_out = smem + L::kOutOffset;
+        const uint32_t acc_empty_rank0 = map_to_rank(acc_empty, 0);
+        uint32_t tcount = 0;
+        for (int tile = pair; tile < n_tiles; tile += n_pairs, ++tcount) {
+            const int tok0 = tile_tok0(tile), count = min(BN, a.M - tok0);
+            const bool got = mbar_wait(acc_full, tcount & 1, abort_flag, a.status, 4);
+            uint32_t gave_up;  // OR over the four epilogue warps, so that they leave together
+            asm volatile(
+                "{\n"
+                ".reg .pred p, q;\n"
+                "setp.ne.u32 q, %1, 0;\n"
+                "bar.red.or.pred p, 2, %2, q;\n"
+                "selp.u32 %0, 1, 0, p;\n"
+                "}\n"
+                : "=r"(gave_up)
+                : "r"(static_cast<uint32_t>(!got)), "n"(kEpiWarps * 32)
+                : "memory");
+            if (gave_up) break;
+            tcgen05_fence_after();
+            const int row_l = quarter * 32 + lane;
+            const int o0 = tile_rows(tile) * BM;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            const int n_half = (count + 127) / 128;
+            for (int hf = 0; hf < n_half; ++hf) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    if (hf * 128 + c0 >= count) break;
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(taddr + hf * 128 + c0, r);
+                    tcgen05_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<__half *>(stage_out + (c0 + j) * 256 + row_l * 2) = __float2half_rn(__uint_as_float(r[j]));
+                }
+                if (hf == n_half - 1) {  // every column of the accumulator has been read
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acc_empty_rank0);
+                }
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                const int n_tok = min(128, count - hf * 128);
+                for (int idx = et; idx < n_tok * 16; idx += kEpiWarps * 32) {
+                    const int tok = idx >> 4, ch = idx & 15;
+                    const int o = o0 + ch * 8;
+                    __half *dst = a.y + static_cast<size_t>(tok0 + hf * 128 + tok) * a.ldy + o;
+                    const uint4 val = *reinterpret_cast<const uint4 *>(stage_out + tok * 256 + ch * 16);
+                    if (a.y_vec_ok && o + 8 <= a.d_out) {
+                        *reinterpret_cast<uint4 *>(dst) = val;
+                    } else {
+                        const __half *hv = reinterpret_cast<const __half *>(&val);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (o + q < a.d_out) dst[q] = hv[q];
+                    }
+                }
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
+            }
+        }
+    } else {
+        // ------------------------------------------------ transform: this CTA's W_b tile -> its W_hat slot, as in the kernel above
+        const int quarter = warp & 3;
+        const uint32_t par = static_cast<uint32_t>((warp - (2 + kEpiWarps)) >> 2);
+        const int r = quarter * 32 + lane;
+        const int words = a.d_in >> 5;
+        const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
+        const uint32_t ready_rank0 = map_to_rank(ready, 0);
+        constexpr bool delta = HAS_DELTA, col = AXIS == PD_AXIS_COL;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+            const int o = tile_rows(tile) * BM + r;
+            const bool row_ok = o < a.d_out;
+            uint32_t vrow = 0;
+            if (delta && !col && row_ok) {
+                const uint32_t hv = *reinterpret_cast<const unsigned short *>(a.v + o);
+                vrow = hv | (hv << 16);
+            }
+            const uint32_t *mrow = delta ? a.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
+            auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
+                w0 = (delta && row_ok && ks < a.k_steps && 2 * ks < words) ? __ldg(mrow + 2 * ks) : 0u;
+                w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
+            };
+            int ks = static_cast<int>((par ^ it) & 1u);
+            uint32_t q0[4], q1[4];
+#pragma unroll
+            for (int d = 0; d < 4; ++d) load_words(ks + 2 * d, q0[d], q1[d]);
+            for (; ks < a.k_steps; ks += 2) {
+                const uint32_t my_it = it + ks;
+                const int s = my_it % L::kStages, sa = my_it % kASlots;
+                const uint32_t word[2] = {q0[0], q1[0]};
+#pragma unroll
+                for (int d = 0; d < 3; ++d) q0[d] = q0[d + 1], q1[d] = q1[d + 1];
+                load_words(ks + 8, q0[3], q1[3]);
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, (my_it / L::kStages) & 1, abort_flag, a.status, 5)))) break;
+                const unsigned char *wt = smem + L::kWOffset + s * L::kWBytes + r * 128;
+                const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
+                uint32_t out[32];
+                build_w_hat_row<delta, delta && col>(out, wt, vs, r, vrow, word[0], word[1]);
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
+                tcgen05_fence_after();
+                tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
+                // all shared-memory reads of the W_b slot have returned once the store has taken its operands
+                __syncwarp();
+                if (lane == 0) mbar_arrive(w_empty + s);
+                tcgen05_wait_st();
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(ready_rank0 + static_cast<uint32_t>(sa) * 8u);
+            }
+            it += a.k_steps;
+        }
+    }
+
+    // ------------------------------------------------ teardown: neither CTA may leave (or free tensor memory) while the
+    // other can still read its shared memory, arrive on its barriers or multiply from its tensor memory
+    tcgen05_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        __syncthreads();
+    }
+    cluster_sync_all();
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        tcgen05_dealloc_pair(tmem_base, 512);
+    }
+}
+
+
 // ------------------------------------------------------------------ host side
 // fp16 row-major [rows, cols] with row pitch ld elements; box = 64 columns x box_rows rows, 128-byte swizzle
 bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
@@ -520,6 +870,61 @@ pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *
 
 }  // namespace
 
+namespace {
+
+template <int AXIS, bool HAS_DELTA>
+pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA>;
+    constexpr int smem = PairLayout::kTotal;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return PD_ERR_CUDA;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kNumThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    count_launch();
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, args));
+}
+
+// Tiles of 256 rows x 256 tokens on pairs of CTAs.
+pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
+                           int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                           cudaStream_t stream) {
+    CUtensorMap mw, mx;
+    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, 128)) return PD_ERR_CUDA;
+    GemmArgs args = {};
+    args.mask = mask;
+    args.v = v;
+    args.y = y;
+    args.ldy = ldy;
+    args.M = static_cast<int>(M);
+    args.d_out = static_cast<int>(d_out);
+    args.d_in = static_cast<int>(d_in);
+    args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
+    args.tiles_n = static_cast<int>((M + 255) / 256);
+    args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
+    args.status = status;
+    args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
+    const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
+    const int pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
+    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false>(mw, mx, args, 2 * pairs, stream);
+    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true>(mw, mx, args, 2 * pairs, stream);
+    return launch_pair_one<PD_AXIS_COL, true>(mw, mx, args, 2 * pairs, stream);
+}
+
+}  // namespace
+
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
                       uint32_t *status, cudaStream_t stream) {
@@ -536,6 +941,9 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
         const int64_t cost = ((tiles + sms - 1) / sms) * (2 * bn > 400 ? 2 * bn : 400);
         if (best_cost < 0 || cost <= best_cost) best = bn, best_cost = cost;
     }
+    static const int use_pair = [] { const char *e = getenv("PD_GEMM_PAIR"); return e ? atoi(e) : 1; }();
+    if (best == 256 && use_pair && d_out >= 256)
+        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
