@@ -319,6 +319,17 @@ def test_prefill_7b_sampled_rows(api, d_out, d_in, m, axis):
     check_prefill(api, layer(d_out, d_in), m, axis, rows=synth.sample_rows(m, n_random=16))
 
 
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in,m", [(1152, 992, 4000), (1100, 1088, 3900), (256, 4096, 37000)])
+def test_prefill_cta_pair_ragged_edges(api, d_out, d_in, m, axis):
+    # sizes that take the 256-row x 256-token tiles of the two-CTA kernel with ragged edges: an odd number of
+    # 128-row tiles (the second CTA of the last pair has no rows at all), rows and tokens that end inside a tile,
+    # a last k step of 32 columns, and one row-tile pair walking many token tiles
+    L = layer(d_out, d_in, seed=5)
+    rows = np.unique(np.concatenate([synth.sample_rows(m, n_random=24), np.arange(m - 130, m), np.arange(120, 136)]))
+    check_prefill(api, L, m, axis, rows=rows)
+
+
 # ------------------------------------------------------------------ multi-variant
 def make_variants(w_b, n_var, seed, mixed_axes=True, axis=ROW):
     d_out, d_in = w_b.shape
