@@ -200,15 +200,13 @@ __device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsig
                 const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
                 vv[0] = t4.x, vv[1] = t4.y, vv[2] = t4.z, vv[3] = t4.w;
             }
-            const uint32_t bits = c < 4 ? word0 : word1;
-            const int j = c & 3;  // byte of the word that belongs to this piece
-            const uint32_t sel = static_cast<uint32_t>(((j | 8) << 4) | (((4 + j) | 8) << 12));
+            // the piece's 8 sign bits are byte c & 3 of its word.  b * 0x8001 puts bit i at i and i + 15, so a left
+            // shift by 15 - 2 pr brings bit 2 pr to bit 15 and bit 2 pr + 1 to bit 31: the signs of halves 2 pr (low)
+            // and 2 pr + 1 (high).  +v where the bit is 1, -v where it is 0.
+            const uint32_t sp = prmt(c < 4 ? word0 : word1, 0u, 0x4440u | static_cast<uint32_t>(c & 3)) * 0x8001u;
 #pragma unroll
-            for (int pr = 0; pr < 4; ++pr) {
-                // halves 2pr (low) and 2pr+1 (high) of the piece: +v where the bit is 1, -v where it is 0
-                const uint32_t rep = prmt(bits << (7 - 2 * pr), bits << (6 - 2 * pr), sel);
-                out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(rep, 0x80008000u, vv[pr]));
-            }
+            for (int pr = 0; pr < 4; ++pr)
+                out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(sp << (15 - 2 * pr), 0x80008000u, vv[pr]));
         } else {  // base only: the tile goes to tensor memory unchanged
 #pragma unroll
             for (int pr = 0; pr < 4; ++pr) out[4 * c + pr] = wp[pr];
@@ -478,12 +476,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
 // (TMA fill, operand read): shared-memory bandwidth, which caps the one-CTA kernel at about two thirds
 // of the tensor peak, is no longer the limit.
 //
-// Rank 0 of the pair issues every MMA.  Barriers that gate it live in rank 0 only:
-//   ready[it % 8]   : 4 transform warps of each CTA (rank 1 arrives remotely) + rank 0's x producer, which also
-//                     announces the bytes of BOTH x halves; rank 1's TMA reports its bytes to rank 0's barrier
+// Rank 0 of the pair issues every MMA: per TWO k steps one wait, eight MMAs and one commit (a wait costs the
+// issuing thread ~110 clocks, a commit ~70, an MMA ~70 against 128 clocks of tensor work: per single k step the
+// thread was the bottleneck).  The k steps of a tile are rounded up to an even number; a step past d_in reads
+// zeros.  Barriers that gate the MMA thread live in rank 0 only:
+//   ready[pair % 4] : 4 transform warps of each CTA for each of the two steps (rank 1 arrives remotely) + rank 0's
+//                     x producer, which also announces the bytes of BOTH x halves of both steps; rank 1's TMA
+//                     reports its bytes to rank 0's barrier
 //   acc_empty       : the 4 epilogue warps of each CTA
 // consumed[] and acc_full exist in both CTAs; one multicast tcgen05.commit arrives on both copies.
 // The W_b ring, its barriers and the transform are per CTA, as in the kernel above.
+constexpr int kPairSlots = kASlots / 2;  // ready / consumed barriers: one per two k steps
 struct PairLayout {
     static constexpr int kStages = 6;             // x ring and W_b ring
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
@@ -607,7 +610,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             mbar_init(w_empty + s, kXformWarps / 2);
         }
         for (int s = 0; s < kASlots; ++s) {
-            mbar_init(ready + s, 2 * (kXformWarps / 2) + 1);  // used in rank 0 only
+            mbar_init(ready + s, 2 * kXformWarps + 1);  // used in rank 0 only: two k steps x two CTAs x four warps + x
             mbar_init(consumed + s, 1);
         }
         mbar_init(acc_full, 1);
@@ -641,18 +644,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                     const int s = it % L::kStages;
                     if (is_x) {
-                        if (it >= static_cast<uint32_t>(L::kStages)) {
-                            const uint32_t prev = it - L::kStages;
-                            if (!(ok = mbar_wait(consumed + prev % kASlots, (prev / kASlots) & 1, abort_flag, a.status, 1))) break;
+                        const uint32_t pi = it >> 1;  // pair of k steps: one ready / consumed barrier for both
+                        if ((it & 1u) == 0) {
+                            if (pi >= static_cast<uint32_t>(L::kStages / 2)) {  // the two x slots were last read by pair pi - 3
+                                const uint32_t prev = pi - L::kStages / 2;
+                                if (!(ok = mbar_wait(consumed + prev % kPairSlots, (prev / kPairSlots) & 1, abort_flag, a.status, 1))) break;
+                            }
+                            if (rank == 0) mbar_arrive_expect_tx(ready + pi % kPairSlots, 4 * L::kXBytes);  // both halves of both steps
                         }
-                        uint64_t *rb = ready + it % kASlots;
-                        if (rank == 0) mbar_arrive_expect_tx(rb, 2 * L::kXBytes);  // both halves report here
-                        tma_load_2d_pair(&map_x, map_to_rank(rb, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
+                        tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
                                          tok0 + 128 * static_cast<int>(rank));
                     } else {
                         const uint32_t parity = ((it / L::kStages) & 1) ^ 1;
                         if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
-                        const uint32_t v_bytes = (HAS_DELTA && AXIS == PD_AXIS_COL) ? static_cast<uint32_t>(min(BK, a.d_in - ks * BK) * 2) : 0u;
+                        const uint32_t v_bytes = (HAS_DELTA && AXIS == PD_AXIS_COL) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ks * BK)) * 2) : 0u;
                         mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
                         tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, tm * BM);
                         if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, a.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
@@ -669,16 +674,20 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
                 if (!(ok = mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
-                for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
-                    const int s = it % L::kStages, sa = it % kASlots;
-                    if (!(ok = mbar_wait(ready + sa, (it / kASlots) & 1, abort_flag, a.status, 3))) break;
+                for (int ks = 0; ks < a.k_steps; ks += 2, it += 2) {
+                    const uint32_t pi = it >> 1;
+                    if (!(ok = mbar_wait(ready + pi % kPairSlots, (pi / kPairSlots) & 1, abort_flag, a.status, 3))) break;
                     tcgen05_fence_after();
-                    const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kXBytes);
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tcgen05_mma_f16_tmem_a_pair(tmem_base, tmem_base + kACol0 + sa * 32 + kk * 8, make_smem_desc(x_addr + kk * 32),
-                                                    idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-                    tcgen05_commit_pair(consumed + sa);
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t x_addr = smem_u32(smem + L::kXOffset + ((it + h) % L::kStages) * L::kXBytes);
+                        const uint32_t a_col = tmem_base + kACol0 + ((it + h) % kASlots) * 32;
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            tcgen05_mma_f16_tmem_a_pair(tmem_base, a_col + kk * 8, make_smem_desc(x_addr + kk * 32), idesc,
+                                                        (ks > 0 || h > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tcgen05_commit_pair(consumed + pi % kPairSlots);  // frees the x slots and the W_hat slots of both steps
                 }
                 if (ok) tcgen05_commit_pair(acc_full);
             }
@@ -785,7 +794,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
                 uint32_t out[32];
                 build_w_hat_row<delta, delta && col>(out, wt, vs, r, vrow, word[0], word[1]);
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
+                const uint32_t pi = my_it >> 1;  // the W_hat slot was last read by pair pi - 4
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + pi % kPairSlots, ((pi / kPairSlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
                 tcgen05_fence_after();
                 tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
                 // all shared-memory reads of the W_b slot have returned once the store has taken its operands
@@ -794,7 +804,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 tcgen05_wait_st();
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(ready_rank0 + static_cast<uint32_t>(sa) * 8u);
+                if (lane == 0) mbar_arrive_cluster(ready_rank0 + (pi % kPairSlots) * 8u);
             }
             it += a.k_steps;
         }
@@ -913,7 +923,7 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.d_in = static_cast<int>(d_in);
     args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
     args.tiles_n = static_cast<int>((M + 255) / 256);
-    args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
+    args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;  // even: the MMA thread works on pairs of k steps
     args.status = status;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
