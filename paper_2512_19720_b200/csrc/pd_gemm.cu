@@ -487,6 +487,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
 // consumed[] and acc_full exist in both CTAs; one multicast tcgen05.commit arrives on both copies.
 // The W_b ring, its barriers and the transform are per CTA, as in the kernel above.
 constexpr int kPairSlots = kASlots / 2;  // ready / consumed barriers: one per two k steps
+constexpr int kPairEpiWarps = 8;
+constexpr int kPairWarps = 2 + kPairEpiWarps + kXformWarps + 1;  // 0 x producer, 1 MMA, 2-9 epilogue, 10-17 transform, 18 W_b producer
+constexpr int kPairThreads = kPairWarps * 32;
 struct PairLayout {
     static constexpr int kStages = 6;             // x ring and W_b ring
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
@@ -585,7 +588,7 @@ __device__ __forceinline__ void tcgen05_mma_f16_tmem_a_pair(uint32_t d_tmem, uin
 }
 
 template <int AXIS, bool HAS_DELTA>
-__global__ void __launch_bounds__(kNumThreads, 1)
+__global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
     constexpr int BN = 256;
@@ -614,7 +617,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             mbar_init(consumed + s, 1);
         }
         mbar_init(acc_full, 1);
-        mbar_init(acc_empty, 2 * kEpiWarps);                   // used in rank 0 only
+        mbar_init(acc_empty, 2 * kPairEpiWarps);               // used in rank 0 only
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -633,7 +636,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     auto tile_rows = [&](int tile) { return (tile / a.tiles_n) * 2 + static_cast<int>(rank); };      // W row tile of 128
     auto tile_tok0 = [&](int tile) { return (tile % a.tiles_n) * BN; };
 
-    if (warp == 0 || warp == kNumWarps - 1) {
+    if (warp == 0 || warp == kPairWarps - 1) {
         // ------------------------------------------------ TMA producers
         if (lane == 0) {
             const bool is_x = warp == 0;
@@ -692,9 +695,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 if (ok) tcgen05_commit_pair(acc_full);
             }
         }
-    } else if (warp < 2 + kEpiWarps) {
+    } else if (warp < 2 + kPairEpiWarps) {
         // ------------------------------------------------ epilogue: this CTA's 128 rows of the accumulator, as in the kernel above
+        // eight warps: two per TMEM lane quarter, each draining half of the columns, so that the accumulator goes
+        // back to the MMA thread in half the time (the tensor cores idle while it is drained)
         const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;
         const int et = threadIdx.x - 2 * 32;
         unsigned char *stage_out = smem + L::kOutOffset;
         const uint32_t acc_empty_rank0 = map_to_rank(acc_empty, 0);
@@ -711,7 +717,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 "selp.u32 %0, 1, 0, p;\n"
                 "}\n"
                 : "=r"(gave_up)
-                : "r"(static_cast<uint32_t>(!got)), "n"(kEpiWarps * 32)
+                : "r"(static_cast<uint32_t>(!got)), "n"(kPairEpiWarps * 32)
                 : "memory");
             if (gave_up) break;
             tcgen05_fence_after();
@@ -721,7 +727,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const int n_half = (count + 127) / 128;
             for (int hf = 0; hf < n_half; ++hf) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < 128; c0 += 32) {
+                for (int c0 = 64 * col_half; c0 < 64 * col_half + 64; c0 += 32) {
                     if (hf * 128 + c0 >= count) break;
                     uint32_t r[32];
                     tcgen05_ld_32x32b_x32(taddr + hf * 128 + c0, r);
@@ -735,9 +741,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(acc_empty_rank0);
                 }
-                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(kPairEpiWarps * 32) : "memory");
                 const int n_tok = min(128, count - hf * 128);
-                for (int idx = et; idx < n_tok * 16; idx += kEpiWarps * 32) {
+                for (int idx = et; idx < n_tok * 16; idx += kPairEpiWarps * 32) {
                     const int tok = idx >> 4, ch = idx & 15;
                     const int o = o0 + ch * 8;
                     __half *dst = a.y + static_cast<size_t>(tok0 + hf * 128 + tok) * a.ldy + o;
@@ -751,13 +757,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             if (o + q < a.d_out) dst[q] = hv[q];
                     }
                 }
-                asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(kPairEpiWarps * 32) : "memory");
             }
         }
     } else {
         // ------------------------------------------------ transform: this CTA's W_b tile -> its W_hat slot, as in the kernel above
         const int quarter = warp & 3;
-        const uint32_t par = static_cast<uint32_t>((warp - (2 + kEpiWarps)) >> 2);
+        const uint32_t par = static_cast<uint32_t>((warp - (2 + kPairEpiWarps)) >> 2);
         const int r = quarter * 32 + lane;
         const int words = a.d_in >> 5;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
@@ -893,7 +899,7 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const Ge
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    cfg.blockDim = dim3(kNumThreads);
+    cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
