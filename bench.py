@@ -41,7 +41,7 @@ MULTI_M = (64, 64 + 4 * 512)
 ROW, COL = 0, 1
 # ncu dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, 4096 x 11008 captures in profiles/
 # (merge: reads only -- half of its writes are still dirty in L2 when the kernel ends)
-NCU_DRAM_RATIO = {"decode": 96.13 / 95.81, "pack": (180.52 + 4.84) / (180.36 + 5.67), "merge": 1.0}
+NCU_DRAM_RATIO = {"decode": 96.18 / 95.81, "pack": (180.52 + 4.84) / (180.36 + 5.67), "merge": 1.0}
 METRIC = "fused delta-linear decode HBM GB/s (7B block sweep, M in {1,4,16}, row+col axes)"
 
 
@@ -355,7 +355,7 @@ def run_ours(args):
                     "algorithmic_flops_per_call": work[section] // calls_per[section],
                     "avg_call_ms": round(sec_ms[section] / calls_per[section], 5),
                     "share_of_step": round(sec_ms[section] / sum(sec_ms.values()), 4)}
-        gemm_roof = tensor("prefill", tfl, "gemm_kernel (tcgen05 prefill)")
+        gemm_roof = tensor("prefill", tfl, "gemm_pair_kernel (tcgen05 prefill on CTA pairs; gemm_kernel at M = 256)")
         cpu = oracle_sample(4, 1) if (world == 1 and not args.no_cpu_baseline) else None
         all_roofs = {"decode": hbm("decode", "gemv_stream_kernel (decode)"), "pack": hbm("pack", "pack_kernel"),
                      "merge": hbm("merge", "merge_kernel"), "multivariant_decode": hbm("multi_decode", "gemm_kernel (grouped, M=64 over 16 variants)"),
