@@ -274,11 +274,11 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
         for (int g = 0; g < V; ++g)
             if (axes[g] == PD_AXIS_COL) col_bits |= 1ull << g;
         st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, tile_table, n_token_tiles,
-                               grouped_token_tile(M, V), xh, ldx, d_in, x_sorted, stream);
+                               grouped_token_tile_for(M, V, d_out), xh, ldx, d_in, x_sorted, stream);
         if (st != PD_OK) return st;
         return launch_gemm_grouped(x_sorted, M, static_cast<const __half *>(w_b), masks, mask_words, vh, v_stride, col_bits,
                                    V, d_out, d_in, static_cast<__half *>(y), ldy, tile_table, n_token_tiles,
-                                   static_cast<int>(M / grouped_token_tile(M, V) + V + 2), grouped_token_tile(M, V), row_index, status,
+                                   static_cast<int>(M / grouped_token_tile_for(M, V, d_out) + V + 2), grouped_token_tile_for(M, V, d_out), row_index, status,
                                    stream);
     }
     st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, nullptr, nullptr, 0, nullptr, 0, 0,

@@ -61,6 +61,12 @@ inline int grouped_token_tile(int64_t M, int V) {
     const int64_t avg = M / (V > 0 ? V : 1);
     return avg <= 48 ? 64 : (avg <= 100 ? 128 : 256);
 }
+// The 256-row x 256-token tiles on CTA pairs are in use (PD_GEMM_PAIR=0 turns them off, for comparisons).
+bool gemm_pair_enabled();
+// Token tile the multi-variant path cuts buckets into: 256 when the pair kernel takes them.
+inline int grouped_token_tile_for(int64_t M, int V, int64_t d_out) {
+    return (gemm_pair_enabled() && d_out >= 256) ? 256 : grouped_token_tile(M, V);
+}
 pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,

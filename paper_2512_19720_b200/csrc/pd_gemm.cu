@@ -587,7 +587,41 @@ __device__ __forceinline__ void tcgen05_mma_f16_tmem_a_pair(uint32_t d_tmem, uin
         : "memory");
 }
 
-template <int AXIS, bool HAS_DELTA>
+// Tile of the pair kernel as one CTA sees it.  `half` = token rows each CTA holds in shared memory (MMA N = 2 half).
+struct PairTile {
+    int tm, tok0, count, half;   // this CTA's W row tile of 128; first token row; valid tokens; tokens per CTA
+    const uint32_t *mask;
+    const __half *v;
+    bool col, delta;
+};
+template <int AXIS, bool HAS_DELTA, bool GROUPED>
+__device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, int n_tt, uint32_t rank) {
+    PairTile t;
+    const int tp = tile / n_tt, tn = tile - tp * n_tt;
+    t.tm = 2 * tp + static_cast<int>(rank);
+    if (!GROUPED) {
+        t.tok0 = tn * 256;
+        t.count = min(256, a.M - t.tok0);
+        t.half = 128;
+        t.mask = a.mask;
+        t.v = a.v;
+        t.col = AXIS == PD_AXIS_COL;
+        t.delta = HAS_DELTA;
+    } else {  // one variant's rows (at most 256), MMA N rounded up to a multiple of 32
+        const int4 e = __ldg(a.tile_table + tn);
+        t.tok0 = e.y;
+        t.count = e.z;
+        t.half = ((e.z + 31) & ~31) >> 1;
+        t.delta = e.x < a.V;
+        const int g = t.delta ? e.x : 0;
+        t.mask = a.mask + static_cast<size_t>(g) * a.mask_stride;
+        t.v = a.v + static_cast<size_t>(g) * a.v_stride;
+        t.col = (a.col_axis_bits >> g) & 1ull;
+    }
+    return t;
+}
+
+template <int AXIS, bool HAS_DELTA, bool GROUPED>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
@@ -605,7 +639,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const uint32_t rank = cluster_ctarank();          // 0 issues the MMAs
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int tiles_m2 = (a.tiles_m + 1) >> 1;        // tiles of 256 rows
-    const int n_tiles = tiles_m2 * a.tiles_n;
+    const int n_tt = GROUPED ? __ldg(a.n_token_tiles) : a.tiles_n;  // token tiles
+    const int n_tiles = tiles_m2 * n_tt;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < L::kStages; ++s) {
@@ -632,9 +667,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // tile -> (256-row tile, token tile); this CTA's 128 rows and 128 tokens
-    auto tile_rows = [&](int tile) { return (tile / a.tiles_n) * 2 + static_cast<int>(rank); };      // W row tile of 128
-    auto tile_tok0 = [&](int tile) { return (tile % a.tiles_n) * BN; };
+    auto tile_of = [&](int tile) { return get_pair_tile<AXIS, HAS_DELTA, GROUPED>(a, tile, n_tt, rank); };
 
     if (warp == 0 || warp == kPairWarps - 1) {
         // ------------------------------------------------ TMA producers
@@ -643,7 +676,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             uint32_t it = 0;
             bool ok = true;
             for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
-                const int tm = tile_rows(tile), tok0 = tile_tok0(tile);
+                const PairTile ti = tile_of(tile);
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                     const int s = it % L::kStages;
                     if (is_x) {
@@ -656,14 +689,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             if (rank == 0) mbar_arrive_expect_tx(ready + pi % kPairSlots, 4 * L::kXBytes);  // both halves of both steps
                         }
                         tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
-                                         tok0 + 128 * static_cast<int>(rank));
+                                         ti.tok0 + ti.half * static_cast<int>(rank));
                     } else {
                         const uint32_t parity = ((it / L::kStages) & 1) ^ 1;
                         if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
-                        const uint32_t v_bytes = (HAS_DELTA && AXIS == PD_AXIS_COL) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ks * BK)) * 2) : 0u;
+                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ks * BK)) * 2) : 0u;
                         mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
-                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, tm * BM);
-                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, a.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
+                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, ti.tm * BM);
+                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
                     }
                 }
             }
@@ -673,8 +706,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, tcount = 0;
             bool ok = true;
-            const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
             for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
+                const int n_mma = 2 * tile_of(tile).half;
+                const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
                 if (!(ok = mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
                 for (int ks = 0; ks < a.k_steps; ks += 2, it += 2) {
@@ -706,7 +740,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const uint32_t acc_empty_rank0 = map_to_rank(acc_empty, 0);
         uint32_t tcount = 0;
         for (int tile = pair; tile < n_tiles; tile += n_pairs, ++tcount) {
-            const int tok0 = tile_tok0(tile), count = min(BN, a.M - tok0);
+            const PairTile ti = tile_of(tile);
+            const int tok0 = ti.tok0, count = ti.count;
             const bool got = mbar_wait(acc_full, tcount & 1, abort_flag, a.status, 4);
             uint32_t gave_up;  // OR over the four epilogue warps, so that they leave together
             asm volatile(
@@ -722,7 +757,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             if (gave_up) break;
             tcgen05_fence_after();
             const int row_l = quarter * 32 + lane;
-            const int o0 = tile_rows(tile) * BM;
+            const int o0 = ti.tm * BM;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const int n_half = (count + 127) / 128;
             for (int hf = 0; hf < n_half; ++hf) {
@@ -746,7 +781,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 for (int idx = et; idx < n_tok * 16; idx += kPairEpiWarps * 32) {
                     const int tok = idx >> 4, ch = idx & 15;
                     const int o = o0 + ch * 8;
-                    __half *dst = a.y + static_cast<size_t>(tok0 + hf * 128 + tok) * a.ldy + o;
+                    const int yr = GROUPED ? __ldg(a.row_index + tok0 + hf * 128 + tok) : tok0 + hf * 128 + tok;
+                    __half *dst = a.y + static_cast<size_t>(yr) * a.ldy + o;
                     const uint4 val = *reinterpret_cast<const uint4 *>(stage_out + tok * 256 + ch * 16);
                     if (a.y_vec_ok && o + 8 <= a.d_out) {
                         *reinterpret_cast<uint4 *>(dst) = val;
@@ -768,18 +804,19 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int words = a.d_in >> 5;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
         const uint32_t ready_rank0 = map_to_rank(ready, 0);
-        constexpr bool delta = HAS_DELTA, col = AXIS == PD_AXIS_COL;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
-            const int o = tile_rows(tile) * BM + r;
+            const PairTile ti = tile_of(tile);
+            const bool delta = ti.delta, col = ti.col;  // compile-time constants in the plain mode
+            const int o = ti.tm * BM + r;
             const bool row_ok = o < a.d_out;
             uint32_t vrow = 0;
             if (delta && !col && row_ok) {
-                const uint32_t hv = *reinterpret_cast<const unsigned short *>(a.v + o);
+                const uint32_t hv = *reinterpret_cast<const unsigned short *>(ti.v + o);
                 vrow = hv | (hv << 16);
             }
-            const uint32_t *mrow = delta ? a.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
+            const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
             auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
                 w0 = (delta && row_ok && ks < a.k_steps && 2 * ks < words) ? __ldg(mrow + 2 * ks) : 0u;
                 w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
@@ -799,7 +836,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 const unsigned char *wt = smem + L::kWOffset + s * L::kWBytes + r * 128;
                 const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
                 uint32_t out[32];
-                build_w_hat_row<delta, delta && col>(out, wt, vs, r, vrow, word[0], word[1]);
+                // specialised bodies: a single body with run-time tests inside the unrolled loop spills
+                if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[0], word[1]);
+                else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[0], word[1]);
                 const uint32_t pi = my_it >> 1;  // the W_hat slot was last read by pair pi - 4
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + pi % kPairSlots, ((pi / kPairSlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
                 tcgen05_fence_after();
@@ -834,6 +874,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 
 
 // ------------------------------------------------------------------ host side
+}  // namespace
+
+bool gemm_pair_enabled() {
+    static const bool on = [] { const char *e = getenv("PD_GEMM_PAIR"); return e ? atoi(e) != 0 : true; }();
+    return on;
+}
+
+namespace {
 // fp16 row-major [rows, cols] with row pitch ld elements; box = 64 columns x box_rows rows, 128-byte swizzle
 bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
     return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, rows, cols, ld * 2, BK, box_rows,
@@ -888,9 +936,9 @@ pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *
 
 namespace {
 
-template <int AXIS, bool HAS_DELTA>
+template <int AXIS, bool HAS_DELTA, bool GROUPED>
 pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
-    auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA>;
+    auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA, GROUPED>;
     constexpr int smem = PairLayout::kTotal;
     static bool configured = false;
     if (!configured) {
@@ -934,9 +982,42 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
     const int pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
-    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false>(mw, mx, args, 2 * pairs, stream);
-    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true>(mw, mx, args, 2 * pairs, stream);
-    return launch_pair_one<PD_AXIS_COL, true>(mw, mx, args, 2 * pairs, stream);
+    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false, false>(mw, mx, args, 2 * pairs, stream);
+    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true, false>(mw, mx, args, 2 * pairs, stream);
+    return launch_pair_one<PD_AXIS_COL, true, false>(mw, mx, args, 2 * pairs, stream);
+}
+
+// Multi-variant: token tiles of at most 256 sorted rows, one variant each.
+pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __half *w_b, const uint32_t *masks,
+                                   int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
+                                   int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
+                                   const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
+                                   cudaStream_t stream) {
+    CUtensorMap mw, mx;
+    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, 128)) return PD_ERR_CUDA;
+    GemmArgs args = {};
+    args.mask = masks;
+    args.v = vs;
+    args.y = y;
+    args.ldy = ldy;
+    args.M = static_cast<int>(M);
+    args.d_out = static_cast<int>(d_out);
+    args.d_in = static_cast<int>(d_in);
+    args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
+    args.tiles_n = 0;
+    args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;
+    args.status = status;
+    args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
+    args.tile_table = tile_table;
+    args.n_token_tiles = n_token_tiles;
+    args.row_index = row_index;
+    args.mask_stride = mask_stride;
+    args.v_stride = v_stride;
+    args.col_axis_bits = col_axis_bits;
+    args.V = V;
+    const int64_t tiles = static_cast<int64_t>((args.tiles_m + 1) / 2) * max_token_tiles;  // upper bound; the kernel reads the real count
+    const int pairs = tiles < sm_count() / 2 ? static_cast<int>(tiles) : sm_count() / 2;
+    return launch_pair_one<PD_AXIS_ROW, true, true>(mw, mx, args, 2 * pairs, stream);
 }
 
 }  // namespace
@@ -957,8 +1038,7 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
         const int64_t cost = ((tiles + sms - 1) / sms) * (2 * bn > 400 ? 2 * bn : 400);
         if (best_cost < 0 || cost <= best_cost) best = bn, best_cost = cost;
     }
-    static const int use_pair = [] { const char *e = getenv("PD_GEMM_PAIR"); return e ? atoi(e) : 1; }();
-    if (best == 256 && use_pair && d_out >= 256)
+    if (best == 256 && gemm_pair_enabled() && d_out >= 256)
         return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
@@ -1007,6 +1087,9 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
                               uint32_t *status, cudaStream_t stream) {
+    if (token_tile == 256 && gemm_pair_enabled() && d_out >= 256)
+        return launch_gemm_pair_grouped(x_sorted, M, w_b, masks, mask_stride, vs, v_stride, col_axis_bits, V, d_out, d_in, y, ldy,
+                                        tile_table, n_token_tiles, max_token_tiles, row_index, status, stream);
 #define PD_GROUPED(BN)                                                                                                     \
     return launch_gemm_grouped_bn<BN>(x_sorted, M, w_b, masks, mask_stride, vs, v_stride, col_axis_bits, V, d_out, d_in, y, \
                                       ldy, tile_table, n_token_tiles, max_token_tiles, row_index, status, stream)
