@@ -487,9 +487,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
 // consumed[] and acc_full exist in both CTAs; one multicast tcgen05.commit arrives on both copies.
 // The W_b ring, its barriers and the transform are per CTA, as in the kernel above.
 constexpr int kPairSlots = kASlots / 2;  // ready / consumed barriers: one per two k steps
-constexpr int kPairEpiWarps = 8;
-constexpr int kPairWarps = 2 + kPairEpiWarps + kXformWarps + 1;  // 0 x producer, 1 MMA, 2-9 epilogue, 10-17 transform, 18 W_b producer
-constexpr int kPairThreads = kPairWarps * 32;
+// warps: 0 x producer, 1 MMA, then the epilogue warps, 8 transform warps, the W_b producer.  Eight epilogue warps
+// for full tiles of 256 tokens; the multi-variant tiles are narrower and the four warps saved leave the
+// transform 128 registers per thread instead of 96 (it spilled there).
+__host__ __device__ constexpr int pair_epi_warps(bool grouped) { return grouped ? 4 : 8; }
+__host__ __device__ constexpr int pair_threads(bool grouped) { return (2 + pair_epi_warps(grouped) + kXformWarps + 1) * 32; }
 struct PairLayout {
     static constexpr int kStages = 6;             // k steps in the x ring and in the W_b ring
     static constexpr int kWPairStages = kStages / 2;  // the W_b ring is filled and freed two k steps at a time
@@ -623,9 +625,10 @@ __device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, i
 }
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED>
-__global__ void __launch_bounds__(kPairThreads, 1)
+__global__ void __launch_bounds__(pair_threads(GROUPED), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
+    constexpr int kEpiW = pair_epi_warps(GROUPED), kWarps = pair_threads(GROUPED) / 32;
     constexpr int BN = 256;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -653,7 +656,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             mbar_init(consumed + s, 1);
         }
         mbar_init(acc_full, 1);
-        mbar_init(acc_empty, 2 * kPairEpiWarps);               // used in rank 0 only
+        mbar_init(acc_empty, 2 * kEpiW);               // used in rank 0 only
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -670,7 +673,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 
     auto tile_of = [&](int tile) { return get_pair_tile<AXIS, HAS_DELTA, GROUPED>(a, tile, n_tt, rank); };
 
-    if (warp == 0 || warp == kPairWarps - 1) {
+    if (warp == 0 || warp == kWarps - 1) {
         // ------------------------------------------------ TMA producers
         if (lane == 0) {
             const bool is_x = warp == 0;
@@ -734,12 +737,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 if (ok) tcgen05_commit_pair(acc_full);
             }
         }
-    } else if (warp < 2 + kPairEpiWarps) {
+    } else if (warp < 2 + kEpiW) {
         // ------------------------------------------------ epilogue: this CTA's 128 rows of the accumulator, as in the kernel above
         // eight warps: two per TMEM lane quarter, each draining half of the columns, so that the accumulator goes
         // back to the MMA thread in half the time (the tensor cores idle while it is drained)
         const int quarter = warp & 3;
         const int col_half = (warp - 2) >> 2;
+        constexpr int kColsPerWarp = 128 / (kEpiW / 4);  // of each half of 128 tokens
         const int et = threadIdx.x - 2 * 32;
         unsigned char *stage_out = smem + L::kOutOffset;
         const uint32_t acc_empty_rank0 = map_to_rank(acc_empty, 0);
@@ -757,7 +761,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 "selp.u32 %0, 1, 0, p;\n"
                 "}\n"
                 : "=r"(gave_up)
-                : "r"(static_cast<uint32_t>(!got)), "n"(kPairEpiWarps * 32)
+                : "r"(static_cast<uint32_t>(!got)), "n"(kEpiW * 32)
                 : "memory");
             if (gave_up) break;
             tcgen05_fence_after();
@@ -767,7 +771,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const int n_half = (count + 127) / 128;
             for (int hf = 0; hf < n_half; ++hf) {
 #pragma unroll 1
-                for (int c0 = 64 * col_half; c0 < 64 * col_half + 64; c0 += 32) {
+                for (int c0 = kColsPerWarp * col_half; c0 < kColsPerWarp * (col_half + 1); c0 += 32) {
                     if (hf * 128 + c0 >= count) break;
                     uint32_t r[32];
                     tcgen05_ld_32x32b_x32(taddr + hf * 128 + c0, r);
@@ -781,9 +785,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(acc_empty_rank0);
                 }
-                asm volatile("bar.sync 2, %0;" ::"n"(kPairEpiWarps * 32) : "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiW * 32) : "memory");
                 const int n_tok = min(128, count - hf * 128);
-                for (int idx = et; idx < n_tok * 16; idx += kPairEpiWarps * 32) {
+                for (int idx = et; idx < n_tok * 16; idx += kEpiW * 32) {
                     const int tok = idx >> 4, ch = idx & 15;
                     const int o = o0 + ch * 8;
                     const int yr = GROUPED ? __ldg(a.row_index + tok0 + hf * 128 + tok) : tok0 + hf * 128 + tok;
@@ -798,13 +802,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             if (o + q < a.d_out) dst[q] = hv[q];
                     }
                 }
-                asm volatile("bar.sync 2, %0;" ::"n"(kPairEpiWarps * 32) : "memory");
+                asm volatile("bar.sync 2, %0;" ::"n"(kEpiW * 32) : "memory");
             }
         }
     } else {
         // ------------------------------------------------ transform: this CTA's W_b tile -> its W_hat slot, as in the kernel above
         const int quarter = warp & 3;
-        const uint32_t grp = static_cast<uint32_t>((warp - (2 + kPairEpiWarps)) >> 2);  // takes the pairs of k steps with pi % 2 == grp
+        const uint32_t grp = static_cast<uint32_t>((warp - (2 + kEpiW)) >> 2);  // takes the pairs of k steps with pi % 2 == grp
         const int r = quarter * 32 + lane;
         const int words = a.d_in >> 5;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
@@ -959,7 +963,7 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const Ge
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    cfg.blockDim = dim3(kPairThreads);
+    cfg.blockDim = dim3(pair_threads(GROUPED));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
