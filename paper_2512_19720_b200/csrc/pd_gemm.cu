@@ -626,8 +626,7 @@ __device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, i
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED>
 __global__ void __launch_bounds__(pair_threads(GROUPED), 1)
-gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                 const __grid_constant__ CUtensorMap map_x64, const __grid_constant__ CUtensorMap map_x32, const GemmArgs a) {
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
     constexpr int kEpiW = pair_epi_warps(GROUPED), kWarps = pair_threads(GROUPED) / 32;
     constexpr int BN = 256;
@@ -691,14 +690,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                                 const uint32_t prev = pi - L::kStages / 2;
                                 if (!(ok = mbar_wait(consumed + prev % kPairSlots, (prev / kPairSlots) & 1, abort_flag, a.status, 1))) break;
                             }
+                            if (rank == 0) mbar_arrive_expect_tx(ready + pi % kPairSlots, 4 * L::kXBytes);  // both halves of both steps
                         }
-                        // multi-variant tiles are often narrow: a box of 32 or 64 token rows instead of 128 spares
-                        // L2 bandwidth, which is what bounds that mode
-                        const int box_rows = (GROUPED && ti.half <= 32) ? 32 : ((GROUPED && ti.half <= 64) ? 64 : 128);
-                        if ((it & 1u) == 0 && rank == 0)
-                            mbar_arrive_expect_tx(ready + pi % kPairSlots, 4u * box_rows * BK * 2);  // both halves of both steps
-                        const CUtensorMap *mx = box_rows == 32 ? &map_x32 : (box_rows == 64 ? &map_x64 : &map_x);
-                        tma_load_2d_pair(mx, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
+                        tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
                                          ti.tok0 + ti.half * static_cast<int>(rank));
                     } else if ((it & 1u) == 0) {
                         // W_b of two k steps (two boxes, 32 KB) and their col-axis scales on one barrier
@@ -959,8 +953,7 @@ pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *
 namespace {
 
 template <int AXIS, bool HAS_DELTA, bool GROUPED>
-pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const CUtensorMap &mx64, const CUtensorMap &mx32,
-                          const GemmArgs &args, int grid, cudaStream_t stream) {
+pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
     auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA, GROUPED>;
     constexpr int smem = PairLayout::kTotal;
     static bool configured = false;
@@ -981,7 +974,7 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const CU
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     count_launch();
-    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, mx64, mx32, args));
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, args));
 }
 
 // Tiles of 256 rows x 256 tokens on pairs of CTAs.
@@ -1005,9 +998,9 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
     const int pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
-    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false, false>(mw, mx, mx, mx, args, 2 * pairs, stream);
-    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true, false>(mw, mx, mx, mx, args, 2 * pairs, stream);
-    return launch_pair_one<PD_AXIS_COL, true, false>(mw, mx, mx, mx, args, 2 * pairs, stream);
+    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false, false>(mw, mx, args, 2 * pairs, stream);
+    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true, false>(mw, mx, args, 2 * pairs, stream);
+    return launch_pair_one<PD_AXIS_COL, true, false>(mw, mx, args, 2 * pairs, stream);
 }
 
 // Multi-variant: token tiles of at most 256 sorted rows, one variant each.
@@ -1016,10 +1009,8 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
                                    int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                                    const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
                                    cudaStream_t stream) {
-    CUtensorMap mw, mx, mx64, mx32;
-    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, 128) ||
-        !make_map(&mx64, x_sorted, M, d_in, d_in, 64) || !make_map(&mx32, x_sorted, M, d_in, d_in, 32))
-        return PD_ERR_CUDA;
+    CUtensorMap mw, mx;
+    if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, 128)) return PD_ERR_CUDA;
     GemmArgs args = {};
     args.mask = masks;
     args.v = vs;
@@ -1042,7 +1033,7 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
     args.V = V;
     const int64_t tiles = static_cast<int64_t>((args.tiles_m + 1) / 2) * max_token_tiles;  // upper bound; the kernel reads the real count
     const int pairs = tiles < sm_count() / 2 ? static_cast<int>(tiles) : sm_count() / 2;
-    return launch_pair_one<PD_AXIS_ROW, true, true>(mw, mx, mx64, mx32, args, 2 * pairs, stream);
+    return launch_pair_one<PD_AXIS_ROW, true, true>(mw, mx, args, 2 * pairs, stream);
 }
 
 }  // namespace
