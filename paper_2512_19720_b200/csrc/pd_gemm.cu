@@ -489,12 +489,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
 constexpr int kPairSlots = kASlots / 2;  // ready / consumed barriers: one per two k steps
 // warps: 0 x producer, 1 MMA, then the epilogue warps, 8 transform warps, the W_b producer.  Eight epilogue warps
 // for full tiles of 256 tokens; the multi-variant tiles are narrower and the four warps saved leave the
-// transform 128 registers per thread instead of 96 (it spilled there).
+// transform 128 registers per thread instead of 96.
 __host__ __device__ constexpr int pair_epi_warps(bool grouped) { return grouped ? 4 : 8; }
 __host__ __device__ constexpr int pair_threads(bool grouped) { return (2 + pair_epi_warps(grouped) + kXformWarps + 1) * 32; }
 struct PairLayout {
-    static constexpr int kStages = 6;             // k steps in the x ring and in the W_b ring
-    static constexpr int kWPairStages = kStages / 2;  // the W_b ring is filled and freed two k steps at a time
+    static constexpr int kStages = 6;             // x ring and W_b ring
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
     static constexpr int kXBytes = 128 * BK * 2;  // this CTA's half of the token tile: 16 KB
     static constexpr int kXOffset = 0;
@@ -503,6 +502,9 @@ struct PairLayout {
     static constexpr int kVOffset = kBarOffset + 512;
     static constexpr int kOutOffset = kVOffset + kStages * kVSlotBytes;
     static constexpr int kTotal = kOutOffset + 128 * 128 * 2 + 1024;
+    // A W_b stage must always fall to the same transform group (even / odd k steps).  Were stages dealt to the
+    // groups in turn, a group could wait for "its" phase of a stage while the other group's phase of that stage is
+    // still in flight, see the parity of the phase before that one and take the stage too early.
     static_assert(kStages % 2 == 0 && kStages <= kASlots, "ring depth");
     static_assert(kTotal <= 227 * 1024, "shared memory per CTA");
 };
@@ -647,12 +649,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const int n_tiles = tiles_m2 * n_tt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < L::kWPairStages; ++s) {
+        for (int s = 0; s < L::kStages; ++s) {
             mbar_init(w_full + s, 1);
-            mbar_init(w_empty + s, kXformWarps / 2);  // the four warps (one per TMEM lane quarter) that own the pair of k steps
+            mbar_init(w_empty + s, kXformWarps / 2);
         }
         for (int s = 0; s < kASlots; ++s) {
-            mbar_init(ready + s, kXformWarps + 1);  // used in rank 0 only: four warps of each CTA + the x producer
+            mbar_init(ready + s, 2 * kXformWarps + 1);  // used in rank 0 only: two k steps x two CTAs x four warps + x
             mbar_init(consumed + s, 1);
         }
         mbar_init(acc_full, 1);
@@ -694,17 +696,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                         }
                         tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
                                          ti.tok0 + ti.half * static_cast<int>(rank));
-                    } else if ((it & 1u) == 0) {
-                        // W_b of two k steps (two boxes, 32 KB) and their col-axis scales on one barrier
-                        const uint32_t pi = it >> 1;
-                        const int ws = pi % L::kWPairStages;
-                        if (!(ok = mbar_wait(w_empty + ws, ((pi / L::kWPairStages) & 1) ^ 1, abort_flag, a.status, 6))) break;
-                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(max(0, min(2 * BK, a.d_in - ks * BK)) * 2) : 0u;
-                        mbar_arrive_expect_tx(w_full + ws, 2 * L::kWBytes + v_bytes);
-                        unsigned char *dst = smem + L::kWOffset + ws * 2 * L::kWBytes;
-                        tma_load_2d(&map_w, w_full + ws, dst, ks * BK, ti.tm * BM);
-                        tma_load_2d(&map_w, w_full + ws, dst + L::kWBytes, (ks + 1) * BK, ti.tm * BM);
-                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + ws * 2 * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + ws);
+                    } else {
+                        const uint32_t parity = ((it / L::kStages) & 1) ^ 1;
+                        if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
+                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ks * BK)) * 2) : 0u;
+                        mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
+                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, ti.tm * BM);
+                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
                     }
                 }
             }
@@ -808,7 +806,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     } else {
         // ------------------------------------------------ transform: this CTA's W_b tile -> its W_hat slot, as in the kernel above
         const int quarter = warp & 3;
-        const uint32_t grp = static_cast<uint32_t>((warp - (2 + kEpiW)) >> 2);  // takes the pairs of k steps with pi % 2 == grp
+        const uint32_t par = static_cast<uint32_t>((warp - (2 + kEpiW)) >> 2);
         const int r = quarter * 32 + lane;
         const int words = a.d_in >> 5;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kACol0;
@@ -826,43 +824,36 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 vrow = hv | (hv << 16);
             }
             const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
-            // the four mask words of the pair of k steps that starts at k step ks
-            auto load_words = [&](int ks, uint32_t (&w)[4]) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) w[q] = (delta && row_ok && ks < a.k_steps && 2 * ks + q < words) ? __ldg(mrow + 2 * ks + q) : 0u;
+            auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
+                w0 = (delta && row_ok && ks < a.k_steps && 2 * ks < words) ? __ldg(mrow + 2 * ks) : 0u;
+                w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
             };
-            int ks = 2 * static_cast<int>((grp ^ (it >> 1)) & 1u);  // first k step of this tile's first pair that falls to this group
-            // mask words of this group's next two pairs, in flight: they come from L2 or HBM
-            uint32_t qa[4], qb[4];
-            load_words(ks, qa);
-            load_words(ks + 4, qb);
-            for (; ks < a.k_steps; ks += 4) {
-                const uint32_t pi = (it + ks) >> 1;
-                const int ws = pi % L::kWPairStages;
-                const uint32_t word[4] = {qa[0], qa[1], qa[2], qa[3]};
+            int ks = static_cast<int>((par ^ it) & 1u);
+            uint32_t q0[4], q1[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) qa[q] = qb[q];
-                load_words(ks + 8, qb);
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + ws, (pi / L::kWPairStages) & 1, abort_flag, a.status, 5)))) break;
+            for (int d = 0; d < 4; ++d) load_words(ks + 2 * d, q0[d], q1[d]);
+            for (; ks < a.k_steps; ks += 2) {
+                const uint32_t my_it = it + ks;
+                const int s = my_it % L::kStages, sa = my_it % kASlots;
+                const uint32_t word[2] = {q0[0], q1[0]};
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const unsigned char *wt = smem + L::kWOffset + (ws * 2 + h) * L::kWBytes + r * 128;
-                    const unsigned char *vs = smem + L::kVOffset + (ws * 2 + h) * kVSlotBytes;
-                    uint32_t out[32];
-                    // specialised bodies: a single body with run-time tests inside the unrolled loop spills
-                    if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[2 * h], word[2 * h + 1]);
-                    else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[2 * h], word[2 * h + 1]);
-                    else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[2 * h], word[2 * h + 1]);
-                    if (h == 0) {  // the two W_hat slots were last read by pair pi - 4
-                        if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + pi % kPairSlots, ((pi / kPairSlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
-                        tcgen05_fence_after();
-                    }
-                    tcgen05_st_32x32b_x32(a_taddr + ((2 * pi + h) % kASlots) * 32, out);
-                }
-                if (!ok) break;
-                // all shared-memory reads of the W_b stage have returned once the stores have taken their operands
+                for (int d = 0; d < 3; ++d) q0[d] = q0[d + 1], q1[d] = q1[d + 1];
+                load_words(ks + 8, q0[3], q1[3]);
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, (my_it / L::kStages) & 1, abort_flag, a.status, 5)))) break;
+                const unsigned char *wt = smem + L::kWOffset + s * L::kWBytes + r * 128;
+                const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
+                uint32_t out[32];
+                // specialised bodies: a single body with run-time tests inside the unrolled loop spills
+                if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[0], word[1]);
+                else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                const uint32_t pi = my_it >> 1;  // the W_hat slot was last read by pair pi - 4
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + pi % kPairSlots, ((pi / kPairSlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
+                tcgen05_fence_after();
+                tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
+                // all shared-memory reads of the W_b slot have returned once the store has taken its operands
                 __syncwarp();
-                if (lane == 0) mbar_arrive(w_empty + ws);
+                if (lane == 0) mbar_arrive(w_empty + s);
                 tcgen05_wait_st();
                 tcgen05_fence_before();
                 __syncwarp();
