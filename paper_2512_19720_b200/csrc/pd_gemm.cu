@@ -62,6 +62,7 @@ struct GemmArgs {
     unsigned long long col_axis_bits;  // bit g set: variant g scales along d_in
     int V;
     int y_vec_ok;  // y is 16-byte aligned and ldy a multiple of 8: rows can be written with 16-byte stores
+    int token_tile;  // pair kernel, one variant: tokens per tile (64, 128 or 256)
 };
 
 struct Tile {
@@ -604,10 +605,10 @@ __device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, i
     PairTile t;
     const int tp = tile / n_tt, tn = tile - tp * n_tt;
     t.tm = 2 * tp + static_cast<int>(rank);
-    if (!GROUPED) {
-        t.tok0 = tn * 256;
-        t.count = min(256, a.M - t.tok0);
-        t.half = 128;
+    if (!GROUPED) {  // MMA N = the tile's tokens rounded up to a multiple of 32
+        t.tok0 = tn * a.token_tile;
+        t.count = min(a.token_tile, a.M - t.tok0);
+        t.half = ((t.count + 31) & ~31) >> 1;
         t.mask = a.mask;
         t.v = a.v;
         t.col = AXIS == PD_AXIS_COL;
@@ -970,7 +971,7 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const Ge
 
 // Tiles of 256 rows x 256 tokens on pairs of CTAs.
 pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
-                           int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
+                           int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, int token_tile, uint32_t *status,
                            cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, 128)) return PD_ERR_CUDA;
@@ -983,7 +984,8 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.d_out = static_cast<int>(d_out);
     args.d_in = static_cast<int>(d_in);
     args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
-    args.tiles_n = static_cast<int>((M + 255) / 256);
+    args.tiles_n = static_cast<int>((M + token_tile - 1) / token_tile);
+    args.token_tile = token_tile;
     args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;  // even: the MMA thread works on pairs of k steps
     args.status = status;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
@@ -1032,12 +1034,31 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
                       uint32_t *status, cudaStream_t stream) {
-    // 256 tokens per tile amortise the W_hat transform best, but with few tokens that leaves most SMs without
+    const int sms = sm_count();
+    if (gemm_pair_enabled() && d_out >= 256) {
+        // CTA pairs, tiles of 256 rows x token_tile tokens.  A pair of k steps costs the issuing thread about 1250
+        // clocks whatever the tile's width (the MMA instruction rate), the tensor cores 4 clocks per token; pick the
+        // width with the fewest rounds x that, ties to the narrower tile (more CTAs stream the weights).
+        static const int forced = [] { const char *e = getenv("PD_GEMM_TOKEN_TILE"); return e ? atoi(e) : 0; }();
+        const int64_t tiles_m2 = (d_out + 2 * BM - 1) / (2 * BM);
+        const int pairs = sms / 2;
+        int best_tt = 256;
+        int64_t best_tt_cost = -1;
+        for (int tt = 256; tt >= 64; tt >>= 1) {
+            const int64_t units = tiles_m2 * ((M + tt - 1) / tt);
+            const int64_t per = 4 * tt + 400 > 1250 ? 4 * tt + 400 : 1250;
+            const int64_t cost = ((units + pairs - 1) / pairs) * per;
+            if (best_tt_cost < 0 || cost <= best_tt_cost) best_tt = tt, best_tt_cost = cost;
+        }
+        if (forced == 64 || forced == 128 || forced == 256) best_tt = forced;
+        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, best_tt, status, stream);
+    }
+    // One CTA per tile (fewer than 256 output rows).  256 tokens per tile amortise the W_hat transform best, but with
+    // few tokens that leaves most SMs without
     // a tile (M = 256 on a 4096-row layer: 32 tiles).  Estimated time = waves x per-stage time, where a stage
     // costs the MMA (2 clocks per token) but never less than the transform/handshake floor; ties go to the
     // smaller tile, which spreads the weight stream over more SMs.
     const int64_t tiles_m = (d_out + BM - 1) / BM;
-    const int sms = sm_count();
     int best = 256;
     int64_t best_cost = -1;
     for (int bn = 256; bn >= 64; bn >>= 1) {
@@ -1045,8 +1066,6 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
         const int64_t cost = ((tiles + sms - 1) / sms) * (2 * bn > 400 ? 2 * bn : 400);
         if (best_cost < 0 || cost <= best_cost) best = bn, best_cost = cost;
     }
-    if (best == 256 && gemm_pair_enabled() && d_out >= 256)
-        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
