@@ -355,7 +355,7 @@ def run_ours(args):
                     "algorithmic_flops_per_call": work[section] // calls_per[section],
                     "avg_call_ms": round(sec_ms[section] / calls_per[section], 5),
                     "share_of_step": round(sec_ms[section] / sum(sec_ms.values()), 4)}
-        gemm_roof = tensor("prefill", tfl, "gemm_pair_kernel (tcgen05 prefill on CTA pairs; gemm_kernel at M = 256)")
+        gemm_roof = tensor("prefill", tfl, "gemm_pair_kernel (tcgen05 prefill on CTA pairs)")
         cpu = oracle_sample(4, 1) if (world == 1 and not args.no_cpu_baseline) else None
         all_roofs = {"decode": hbm("decode", "gemv_stream_kernel (decode)"), "pack": hbm("pack", "pack_kernel"),
                      "merge": hbm("merge", "merge_kernel"), "multivariant_decode": hbm("multi_decode", "gemm_kernel (grouped, M=64 over 16 variants)"),
