@@ -314,7 +314,9 @@ def test_prefill_7b_m256_full(api, axis):
 
 
 @pytest.mark.parametrize("axis", [ROW, COL])
-@pytest.mark.parametrize("d_out,d_in,m", [(4096, 4096, 2048), (11008, 4096, 2048), (4096, 11008, 2048), (4096, 4096, 8192)])
+# (4096, 4096, 512) takes 128-token tiles, (11008, 4096, 256) one 256-token tile per pair of CTAs, the others full 256-token tiles
+@pytest.mark.parametrize("d_out,d_in,m", [(4096, 4096, 2048), (11008, 4096, 2048), (4096, 11008, 2048), (4096, 4096, 8192),
+                                          (4096, 4096, 512), (11008, 4096, 256)])
 def test_prefill_7b_sampled_rows(api, d_out, d_in, m, axis):
     check_prefill(api, layer(d_out, d_in), m, axis, rows=synth.sample_rows(m, n_random=16))
 
