@@ -1,5 +1,9 @@
 // Prefill path: Y[M, d_out] = X . (W_b + v (.) B)^T on the 5th-generation tensor cores.
 //
+// Two kernels share this file: gemm_pair_kernel (further down: tiles of 256 output rows on pairs of CTAs with
+// tcgen05.mma.cta_group::2; every layer with at least 256 output rows) and gemm_kernel (one CTA per tile of 128 rows,
+// described first; smaller layers).  Both form W_hat in tensor memory:
+//
 // The MMA computes the transposed tile  D[128 output rows, BN tokens] = W_hat_tile . X_tile^T :
 //   A operand = W_hat tile, 128 rows x 64 k, in TENSOR MEMORY (row = lane, two fp16 per 32-bit column)
 //   B operand = X tile, BN tokens x 64 k, K-major, 128-byte swizzle, in shared memory
@@ -111,16 +115,6 @@ __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fe
 __device__ __forceinline__ void tcgen05_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
-}
-__device__ __forceinline__ void tcgen05_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                                uint32_t accumulate) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
 }
 __device__ __forceinline__ void tcgen05_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -528,37 +522,10 @@ __device__ __forceinline__ uint32_t map_to_rank(const void *p, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
-        "selp.b32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// mbar_wait for a barrier that the other CTA of the pair arrives on
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
-                                                  uint32_t where) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
-    int spins = 0;
-    while (true) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((++spins & 63) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
-                *abort_flag = 1;
-                latch_error(status, PD_ERR_DEVICE_TIMEOUT, where);
-                return false;
-            }
-        }
-    }
-}
+// The waits on barriers that the other CTA arrives on are the plain mbar_wait: the operands the MMA reads travel
+// through the async proxy (TMA, tcgen05.st + fences), and cluster-scoped acquire/release qualifiers on the per-step
+// barrier operations cost 30 % of the kernel's throughput.
+
 // x half of this CTA; the bytes are reported to the barrier at `bar_cluster_addr` (rank 0's)
 __device__ __forceinline__ void tma_load_2d_pair(const CUtensorMap *map, uint32_t bar_cluster_addr, void *dst, int c0, int c1) {
     asm volatile(
@@ -632,7 +599,6 @@ __global__ void __launch_bounds__(pair_threads(GROUPED), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
     constexpr int kEpiW = pair_epi_warps(GROUPED), kWarps = pair_threads(GROUPED) / 32;
-    constexpr int BN = 256;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
