@@ -332,6 +332,22 @@ def test_prefill_cta_pair_ragged_edges(api, d_out, d_in, m, axis):
     check_prefill(api, L, m, axis, rows=rows)
 
 
+@pytest.mark.parametrize("axis", [ROW, COL])
+@pytest.mark.parametrize("d_out,d_in,m", [(256, 160, 17), (257, 96, 33), (383, 992, 64), (385, 224, 65), (512, 64, 129),
+                                          (300, 2080, 255), (640, 128, 257), (1100, 1088, 31)])
+def test_linear_tensor_core_edge_sizes(api, d_out, d_in, m, axis):
+    # the smallest layers that take the two-CTA tiles (256 rows and up), with row counts on both sides of a 128-row
+    # tile, token counts on both sides of the 32-token MMA granule and of the 64/128/256-token tiles, one and two
+    # k steps, an odd number of k steps (padded to even) and a last k step of 32 columns; checked on every output
+    L = layer(d_out, d_in, seed=11)
+    check_prefill(api, L, m, axis)
+    x = synth.gen_x(m, d_in, 77)
+    y = api.pd_linear(dev(x), L.d_w_b, None, None, ROW)  # base only through the same tiles
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == 0
+    assert rel_err(host(y), x.astype(np.float64) @ L.w_b.astype(np.float64).T) <= TOL
+
+
 # ------------------------------------------------------------------ multi-variant
 def make_variants(w_b, n_var, seed, mixed_axes=True, axis=ROW):
     d_out, d_in = w_b.shape
