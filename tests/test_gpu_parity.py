@@ -390,7 +390,9 @@ def test_multivariant_small(api, d_out, d_in, n_var, m):
         assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
 
 
-@pytest.mark.parametrize("d_out,d_in,n_var,m", [(256, 512, 5, 300), (200, 1152, 3, 150), (1024, 1024, 16, 2112), (130, 96, 2, 700)])
+# (384, 320, 2, 700) and (640, 992, 3, 1000): buckets of more than 256 rows are cut into several tiles of the two-CTA kernel
+@pytest.mark.parametrize("d_out,d_in,n_var,m", [(256, 512, 5, 300), (200, 1152, 3, 150), (1024, 1024, 16, 2112), (130, 96, 2, 700),
+                                                (384, 320, 2, 700), (640, 992, 3, 1000)])
 def test_multivariant_prefill_sized(api, d_out, d_in, n_var, m):
     # more than 64 rows: rows are bucketed by variant and run through the grouped tensor-core kernel
     w_b = synth.gen_base(d_out, d_in, 21)
