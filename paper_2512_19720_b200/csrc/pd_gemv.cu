@@ -257,7 +257,9 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 // Eight consumer warps share every step: each takes one 64-column block and all 16 rows.  W_b, mask
 // and the col-axis scales come from shared memory; the x fragments are read straight from global
 // memory -- x is small and L2-resident, and keeping it out of shared memory leaves the ring to the
-// weights.  The delta term enters the same accumulator as x . (+-s) with s = v[row] (row axis) or
+// weights.  With more than 8 tokens the token index is the MMA's M (16) and 8 rows its N; with up to 8
+// tokens the 16 rows are M and the tokens N, which halves the number of MMAs.  The delta term enters
+// the same accumulator as x . (+-s) with s = v[row] (row axis) or
 // s = v[k] (col axis): exact fp16 products summed in fp32 either way.  The eight warps' partial
 // sums are added in warp order through shared memory.
 //
@@ -431,22 +433,45 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     // read from the stage (all lanes with the same t read the same 16 bytes: a broadcast)
                     uint4 vv = make_uint4(0, 0, 0, 0);
                     if (kCol) vv = *reinterpret_cast<const uint4 *>(stage + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
-#pragma unroll
-                    for (int j = 0; j < kTiles; ++j) {
-                        const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
-                        mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                        mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                    if (M16) {
+    #pragma unroll
+                        for (int j = 0; j < kTiles; ++j) {
+                            const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
+                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                            if (HAS_DELTA) {
+                                // the piece's 8 sign bits are byte t of word c.  b * 0x8001 puts bit i at i and i + 15,
+                                // so a left shift by 15 - 2r brings bit 2r to bit 15 and bit 2r + 1 to bit 31: the signs
+                                // of halves 2r, 2r + 1.  A clear bit (B = -1) flips the sign of the magnitude.
+                                const uint32_t sp = prmt(c ? mw[j].y : mw[j].x, 0u, byte_t) * 0x8001u;
+                                const uint32_t pm0 = lop3_andn_xor(sp << 15, 0x80008000u, kCol ? vv.x : mag[j]);
+                                const uint32_t pm1 = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
+                                const uint32_t pm2 = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
+                                const uint32_t pm3 = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
+                                mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm0, pm1);
+                                mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm2, pm3);
+                            }
+                        }
+                    } else {
+                        // up to 8 tokens: the 16 rows are the MMA's M and the tokens its N, so one MMA does what two
+                        // do above (A = the W_b pieces of rows g and g + 8, B = token g's piece of x);
+                        // acc[0] = {row g: tokens 2t, 2t+1; row g + 8: tokens 2t, 2t+1}
+                        const uint4 w0 = *reinterpret_cast<const uint4 *>(box + g * 512 + in_row);
+                        const uint4 w1 = *reinterpret_cast<const uint4 *>(box + (8 + g) * 512 + in_row);
+                        mma16816(acc[0], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
+                        mma16816(acc[0], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
                         if (HAS_DELTA) {
-                            // the piece's 8 sign bits are byte t of word c.  b * 0x8001 puts bit i at i and i + 15,
-                            // so a left shift by 15 - 2r brings bit 2r to bit 15 and bit 2r + 1 to bit 31: the signs
-                            // of halves 2r, 2r + 1.  A clear bit (B = -1) flips the sign of the magnitude.
-                            const uint32_t sp = prmt(c ? mw[j].y : mw[j].x, 0u, byte_t) * 0x8001u;
-                            const uint32_t pm0 = lop3_andn_xor(sp << 15, 0x80008000u, kCol ? vv.x : mag[j]);
-                            const uint32_t pm1 = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
-                            const uint32_t pm2 = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
-                            const uint32_t pm3 = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
-                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm0, pm1);
-                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm2, pm3);
+                            uint32_t pm[2][4];
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {  // sign expansion as above
+                                const uint32_t sp = prmt(c ? mw[j].y : mw[j].x, 0u, byte_t) * 0x8001u;
+                                pm[j][0] = lop3_andn_xor(sp << 15, 0x80008000u, kCol ? vv.x : mag[j]);
+                                pm[j][1] = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
+                                pm[j][2] = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
+                                pm[j][3] = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
+                            }
+                            mma16816(acc[0], pm[0][0], pm[1][0], pm[0][1], pm[1][1], xa.x, xa.y);
+                            mma16816(acc[0], pm[0][2], pm[1][2], pm[0][3], pm[1][3], xa.z, xa.w);
                         }
                     }
                 }
@@ -475,16 +500,24 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             : "memory");
         if (!gave_up) {
             float *mine = red + warp * 16 * R;  // [16 tokens][R rows]
+            if (M16) {
 #pragma unroll
-            for (int j = 0; j < kTiles; ++j)
+                for (int j = 0; j < kTiles; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int ol = 8 * j + 2 * t + e;
+                        mine[g * R + ol] = acc[j][e];
+                        mine[(g + 8) * R + ol] = acc[j][2 + e];
+                    }
+            } else {  // tokens 2t, 2t + 1 of rows g and g + 8
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const int ol = 8 * j + 2 * t + e;
-                    mine[g * R + ol] = acc[j][e];
-                    mine[(g + 8) * R + ol] = acc[j][2 + e];
+                    mine[(2 * t + e) * R + g] = acc[0][e];
+                    mine[(2 * t + e) * R + g + 8] = acc[0][2 + e];
                 }
+            }
             asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
-            for (int idx = threadIdx.x; idx < 16 * R; idx += kStreamConsumers * 32) {  // (token, row) pairs
+            for (int idx = threadIdx.x; idx < (M16 ? 16 : 8) * R; idx += kStreamConsumers * 32) {  // (token, row) pairs
                 const int tok = idx / R, ol = idx % R;
                 float sum = 0.f;
 #pragma unroll
