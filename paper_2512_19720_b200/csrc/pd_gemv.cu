@@ -258,9 +258,9 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
 // and the col-axis scales come from shared memory; the x fragments are read straight from global
 // memory -- x is small and L2-resident, and keeping it out of shared memory leaves the ring to the
 // weights.  With more than 8 tokens the token index is the MMA's M (16) and 8 rows its N; with up to 8
-// tokens the 16 rows are M and the tokens N, which halves the number of MMAs.  The delta term enters
-// the same accumulator as x . (+-s) with s = v[row] (row axis) or
-// s = v[k] (col axis): exact fp16 products summed in fp32 either way.  The eight warps' partial
+// tokens the 16 rows are M and the tokens N, which halves the number of MMAs.  W_hat = W_b +- s with
+// s = v[row] (row axis) or s = v[k] (col axis) is formed in fp16 registers (add.f16x2: one rounding,
+// as the merge and the prefill path form it) and multiplied with fp32 accumulation.  The eight warps' partial
 // sums are added in warp order through shared memory.
 //
 // Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the stream,
@@ -436,9 +436,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     if (M16) {
     #pragma unroll
                         for (int j = 0; j < kTiles; ++j) {
-                            const uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
-                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                            uint4 w = *reinterpret_cast<const uint4 *>(box + (8 * j + g) * 512 + in_row);
                             if (HAS_DELTA) {
                                 // the piece's 8 sign bits are byte t of word c.  b * 0x8001 puts bit i at i and i + 15,
                                 // so a left shift by 15 - 2r brings bit 2r to bit 15 and bit 2r + 1 to bit 31: the signs
@@ -448,18 +446,20 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 const uint32_t pm1 = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
                                 const uint32_t pm2 = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
                                 const uint32_t pm3 = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
-                                mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, pm0, pm1);
-                                mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, pm2, pm3);
+                                // W_hat = W_b +- v in fp16, as the merge and the prefill path form it: one MMA per
+                                // 16 columns instead of one for W_b and one for the signs
+                                w.x = hadd2_u32(w.x, pm0), w.y = hadd2_u32(w.y, pm1);
+                                w.z = hadd2_u32(w.z, pm2), w.w = hadd2_u32(w.w, pm3);
                             }
+                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
                         }
                     } else {
                         // up to 8 tokens: the 16 rows are the MMA's M and the tokens its N, so one MMA does what two
                         // do above (A = the W_b pieces of rows g and g + 8, B = token g's piece of x);
                         // acc[0] = {row g: tokens 2t, 2t+1; row g + 8: tokens 2t, 2t+1}
-                        const uint4 w0 = *reinterpret_cast<const uint4 *>(box + g * 512 + in_row);
-                        const uint4 w1 = *reinterpret_cast<const uint4 *>(box + (8 + g) * 512 + in_row);
-                        mma16816(acc[0], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
-                        mma16816(acc[0], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
+                        uint4 w0 = *reinterpret_cast<const uint4 *>(box + g * 512 + in_row);
+                        uint4 w1 = *reinterpret_cast<const uint4 *>(box + (8 + g) * 512 + in_row);
                         if (HAS_DELTA) {
                             uint32_t pm[2][4];
 #pragma unroll
@@ -470,9 +470,13 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 pm[j][2] = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
                                 pm[j][3] = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
                             }
-                            mma16816(acc[0], pm[0][0], pm[1][0], pm[0][1], pm[1][1], xa.x, xa.y);
-                            mma16816(acc[0], pm[0][2], pm[1][2], pm[0][3], pm[1][3], xa.z, xa.w);
+                            w0.x = hadd2_u32(w0.x, pm[0][0]), w0.y = hadd2_u32(w0.y, pm[0][1]);
+                            w0.z = hadd2_u32(w0.z, pm[0][2]), w0.w = hadd2_u32(w0.w, pm[0][3]);
+                            w1.x = hadd2_u32(w1.x, pm[1][0]), w1.y = hadd2_u32(w1.y, pm[1][1]);
+                            w1.z = hadd2_u32(w1.z, pm[1][2]), w1.w = hadd2_u32(w1.w, pm[1][3]);
                         }
+                        mma16816(acc[0], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
+                        mma16816(acc[0], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
                     }
                 }
             }
