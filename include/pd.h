@@ -92,10 +92,11 @@ pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t
  *   v    : in,  fp16, d_out entries (PD_AXIS_ROW) or d_in entries (PD_AXIS_COL)
  *   y    : out, fp16 [M, d_out], row stride ldy elements
  *
- * fp16 products, fp32 accumulation, one rounding to fp16 at the end.  M <= 16 runs the
- * bandwidth-bound decode kernel, larger M is cut into chunks of 16 rows up to a crossover and
- * runs the tensor-core (tcgen05) kernel beyond it.  The tensor-core kernel needs d_out and
- * d_in to be multiples of 8 and d_in >= 64.  Needs pd_workspace_bytes(PD_OP_LINEAR, M, ...).
+ * W_hat = W_b +- v is formed on chip in fp16 (one rounding per weight, as pd_merge stores it),
+ * products are accumulated in fp32 and y is rounded to fp16 once at the end.  M <= 16 runs the
+ * bandwidth-bound decode kernel, larger M the tensor-core (tcgen05) kernel, which needs d_out and
+ * d_in to be multiples of 8 and d_in >= 64 (otherwise the rows go through the decode kernel in
+ * chunks of 16).  Needs pd_workspace_bytes(PD_OP_LINEAR, M, ...).
  */
 pd_status pd_linear(const void *x, int64_t M, int64_t ldx,
                     const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
