@@ -457,7 +457,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     } else {
                         // up to 8 tokens: the 16 rows are the MMA's M and the tokens its N, so one MMA does what two
                         // do above (A = the W_b pieces of rows g and g + 8, B = token g's piece of x);
-                        // acc[0] = {row g: tokens 2t, 2t+1; row g + 8: tokens 2t, 2t+1}
+                        // acc[c] = {row g: tokens 2t, 2t+1; row g + 8: tokens 2t, 2t+1}
                         uint4 w0 = *reinterpret_cast<const uint4 *>(box + g * 512 + in_row);
                         uint4 w1 = *reinterpret_cast<const uint4 *>(box + (8 + g) * 512 + in_row);
                         if (HAS_DELTA) {
@@ -475,8 +475,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             w1.x = hadd2_u32(w1.x, pm[1][0]), w1.y = hadd2_u32(w1.y, pm[1][1]);
                             w1.z = hadd2_u32(w1.z, pm[1][2]), w1.w = hadd2_u32(w1.w, pm[1][3]);
                         }
-                        mma16816(acc[0], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
-                        mma16816(acc[0], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
+                        // the two pieces of a block go to accumulators of their own: two short chains of dependent MMAs
+                        mma16816(acc[c], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
+                        mma16816(acc[c], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
                     }
                 }
             }
@@ -516,8 +517,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             } else {  // tokens 2t, 2t + 1 of rows g and g + 8
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    mine[(2 * t + e) * R + g] = acc[0][e];
-                    mine[(2 * t + e) * R + g + 8] = acc[0][2 + e];
+                    mine[(2 * t + e) * R + g] = acc[0][e] + acc[1][e];
+                    mine[(2 * t + e) * R + g + 8] = acc[0][2 + e] + acc[1][2 + e];
                 }
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kStreamConsumers * 32) : "memory");
