@@ -58,6 +58,18 @@ __device__ __forceinline__ uint32_t abs_diff_units_small(float a, float b) {
     return __float_as_uint(fabsf(__fsub_rn(a, b)) + 0.5f) - 0x3f000000u;
 }
 
+// Programmatic dependent launch: a pack call is three kernels (zero the sums, pack, finalize).  Each lets the
+// next one be scheduled as soon as it has started and the next one waits for it before it touches the sums, so
+// the launch latencies overlap the kernels instead of adding to them.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__global__ void zero_sums_kernel(unsigned long long *__restrict__ sums, int n) {
+    grid_launch_dependents();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) sums[i] = 0ull;
+}
+
 template <bool ROW, bool COL>
 __global__ void __launch_bounds__(kThreads)
 pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_out, int d_in, int tiles_c,
@@ -74,6 +86,7 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
     uint32_t cacc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) cacc[j] = 0;
+    grid_launch_dependents();  // the finalize kernel may be scheduled; it waits for this grid
 
 #pragma unroll 4
     for (int rr = warp; rr < kTileRows; rr += kThreads / 32) {
@@ -82,9 +95,14 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
         uint32_t bits = 0, fast_sum = 0;
         unsigned long long slow_sum = 0;
         bool slow = false;
+        uint4 a4 = make_uint4(0, 0, 0, 0), b4 = a4;
         if (col_ok) {
             const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
-            const uint4 a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
+            a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
+        }
+        // the first loads are in flight; nothing may be added to the sums before the kernel that zeroes them is done
+        if (rr == warp) grid_dependency_wait();
+        if (col_ok) {
             const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
             uint32_t spread = 0, u[8], u_or = 0;
 #pragma unroll
@@ -140,6 +158,7 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
             if (lane == 0) atomicAdd(row_sum + o, total);
         }
     }
+    grid_dependency_wait();  // warps without a row in this tile have not waited yet
     if (COL) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) s_col[warp * kTileCols + lane * 8 + j] = cacc[j];
@@ -158,6 +177,7 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
 __global__ void pack_finalize_kernel(const unsigned long long *__restrict__ row_sum,
                                      const unsigned long long *__restrict__ col_sum, int d_out, int d_in,
                                      __half *__restrict__ v_row, __half *__restrict__ v_col) {
+    grid_dependency_wait();  // every tile has added its sums
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     const bool is_row = idx < d_out;
     const int j = is_row ? idx : idx - d_out;
@@ -225,22 +245,35 @@ merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *
 pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
                       __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream) {
     unsigned long long *row_sum = sums, *col_sum = sums + d_out;
-    if (cudaMemsetAsync(sums, 0, sizeof(unsigned long long) * static_cast<size_t>(d_out + d_in), stream) != cudaSuccess)
-        return PD_ERR_CUDA;
+    const int n = static_cast<int>(d_out + d_in);
+    zero_sums_kernel<<<(n + 255) / 256, 256, 0, stream>>>(sums, n);
     const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
     const int64_t tiles = ((d_out + kTileRows - 1) / kTileRows) * tiles_c;
-    const dim3 grid(static_cast<unsigned>(tiles)), block(kThreads);
     const uint4 *a = reinterpret_cast<const uint4 *>(w_f), *b = reinterpret_cast<const uint4 *>(w_b);
     const int n_out = static_cast<int>(d_out), n_in = static_cast<int>(d_in);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled while the previous kernel runs
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles));
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
     if (v_row && v_col)
-        pack_kernel<true, true><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+        e = cudaLaunchKernelEx(&cfg, pack_kernel<true, true>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
     else if (v_row)
-        pack_kernel<true, false><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+        e = cudaLaunchKernelEx(&cfg, pack_kernel<true, false>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
     else
-        pack_kernel<false, true><<<grid, block, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    const int n = static_cast<int>(d_out + d_in);
-    pack_finalize_kernel<<<(n + 255) / 256, 256, 0, stream>>>(row_sum, col_sum, n_out, n_in, v_row, v_col);
-    count_launch(2);
+        e = cudaLaunchKernelEx(&cfg, pack_kernel<false, true>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    if (e != cudaSuccess) return PD_ERR_CUDA;
+    cfg.gridDim = dim3(static_cast<unsigned>((n + 255) / 256));
+    cfg.blockDim = dim3(256);
+    if (cudaLaunchKernelEx(&cfg, pack_finalize_kernel, static_cast<const unsigned long long *>(row_sum),
+                           static_cast<const unsigned long long *>(col_sum), n_out, n_in, v_row, v_col) != cudaSuccess)
+        return PD_ERR_CUDA;
+    count_launch(3);
     return cuda_ok(cudaGetLastError());
 }
 
