@@ -41,7 +41,7 @@ MULTI_M = (64, 64 + 4 * 512)
 ROW, COL = 0, 1
 # ncu dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes, 4096 x 11008 captures in profiles/
 # (merge: reads only -- half of its writes are still dirty in L2 when the kernel ends)
-NCU_DRAM_RATIO = {"decode": 96.19 / 95.81, "pack": (180.52 + 4.84) / (180.36 + 5.67), "merge": 1.0}
+NCU_DRAM_RATIO = {"decode": 96.19 / 95.81, "pack": (180.52 + 4.82) / (180.36 + 5.67), "merge": 1.0}
 METRIC = "fused delta-linear decode HBM GB/s (7B block sweep, M in {1,4,16}, row+col axes)"
 
 
