@@ -1,7 +1,6 @@
 // C ABI of the pd library: argument checks, workspace layout, dispatch.  No device memory is
 // allocated here; everything runs on the caller's stream.
 #include <climits>
-#include <cstdlib>
 
 #include "pd_common.cuh"
 
@@ -92,11 +91,12 @@ group_rows_kernel(const int32_t *__restrict__ ids, int M, int V, int *__restrict
     }
 }
 
-// x_sorted[i, :] = x[row_index[i], :], 16 bytes per thread
+// x_sorted[i, :] = x[row_index[i], :], 16 bytes per thread.  Only the first *n_valid entries of row_index exist
+// (rows with an id outside [-1, V) are in no bucket); the rows of x_sorted past them belong to no token tile.
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(const __half *__restrict__ x, int64_t ldx, int M, int vec_per_row, const int *__restrict__ row_index,
-                   uint4 *__restrict__ x_sorted) {
-    const int64_t total = static_cast<int64_t>(M) * vec_per_row;
+gather_rows_kernel(const __half *__restrict__ x, int64_t ldx, const int *__restrict__ n_valid, int vec_per_row,
+                   const int *__restrict__ row_index, uint4 *__restrict__ x_sorted) {
+    const int64_t total = static_cast<int64_t>(*n_valid) * vec_per_row;
     for (int64_t i = blockIdx.x * 256ll + threadIdx.x; i < total; i += gridDim.x * 256ll) {
         const int r = static_cast<int>(i / vec_per_row), c = static_cast<int>(i - static_cast<int64_t>(r) * vec_per_row);
         x_sorted[i] = *reinterpret_cast<const uint4 *>(x + static_cast<size_t>(row_index[r]) * ldx + 8 * c);
@@ -124,7 +124,7 @@ pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int 
         const int vec_per_row = static_cast<int>(d_in / 8);
         const int64_t blocks = (static_cast<int64_t>(M) * vec_per_row + 255) / 256;
         gather_rows_kernel<<<static_cast<unsigned>(blocks < 4096 ? blocks : 4096), 256, 0, stream>>>(
-            x, ldx, M, vec_per_row, row_index, reinterpret_cast<uint4 *>(x_sorted));
+            x, ldx, offsets + V + 1, vec_per_row, row_index, reinterpret_cast<uint4 *>(x_sorted));
         count_launch();
     }
     return cuda_ok(cudaGetLastError());
@@ -150,8 +150,10 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
             return kStatusBytes;
         case PD_OP_LINEAR_MULTIVARIANT:
             if (M <= 0 || V <= 0) return kStatusBytes + kOffsetsBytes;
+            if (M <= kMvDecodeMaxTokens && d_in % 128 == 0)  // decode batches: x (and col-axis scales) re-laid out
+                return kStatusBytes + mv_decode_scratch_bytes(M, V, d_in);
             return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256) +
-                   (M > 16 ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
+                   (M > kGemvMaxTokens ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
         case PD_OP_MERGE:
         default:
             return 0;
@@ -263,16 +265,19 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
     const __half *xh = static_cast<const __half *>(x);
     const __half *vh = static_cast<const __half *>(vs);
     const int64_t mask_words = d_out * (d_in / 32);
-    static const int grouped_min = [] { const char *e = getenv("PD_GROUPED_MIN_M"); return e ? atoi(e) : 17; }();
-    if (M >= grouped_min && d_in >= 64) {
+    unsigned long long col_bits = 0;
+    for (int g = 0; g < V; ++g)
+        if (axes[g] == PD_AXIS_COL) col_bits |= 1ull << g;
+    if (M <= kMvDecodeMaxTokens && d_in % 128 == 0)
+        // a decode batch: one launch that streams W_b once and applies every variant's mask to its few rows
+        return launch_mv_decode(xh, static_cast<int>(M), ldx, variant_ids, static_cast<const __half *>(w_b), masks, mask_words, vh,
+                                v_stride, col_bits, V, d_out, d_in, static_cast<__half *>(y), ldy, base + kStatusBytes, status, stream);
+    if (M > kGemvMaxTokens && d_in >= 64) {
         // more than one decode chunk: sort the rows by variant, gather them, one grouped tensor-core launch
         unsigned char *p = base + kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256);
         int4 *tile_table = reinterpret_cast<int4 *>(p);
         int *n_token_tiles = reinterpret_cast<int *>(p + grouped_table_bytes(M, V) - 256);
         __half *x_sorted = reinterpret_cast<__half *>(p + grouped_table_bytes(M, V));
-        unsigned long long col_bits = 0;
-        for (int g = 0; g < V; ++g)
-            if (axes[g] == PD_AXIS_COL) col_bits |= 1ull << g;
         st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, tile_table, n_token_tiles,
                                grouped_token_tile_for(M, V, d_out), xh, ldx, d_in, x_sorted, stream);
         if (st != PD_OK) return st;

@@ -25,6 +25,37 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 inline pd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PD_OK : PD_ERR_CUDA; }
 
+// Per-device host state: a process may drive several GPUs from several threads.
+constexpr int kMaxDevices = 64;
+
+inline int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    return dev;
+}
+
+// SM count of the current device.
+inline int sm_count() {
+    static std::atomic<int> cached[kMaxDevices];
+    const int dev = current_device();
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
+// Opts a kernel into `bytes` of dynamic shared memory on the current device, once per device.  The attribute
+// is per device; `done` is the caller's array of kMaxDevices flags for this kernel (one per instantiation).
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<bool> *done) {
+    const int dev = current_device();
+    if (done[dev].load(std::memory_order_acquire)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done[dev].store(true, std::memory_order_release);  // setting it twice from two threads is harmless
+    return true;
+}
+
 __device__ __forceinline__ void latch_error(uint32_t *status, uint32_t code, uint32_t detail) {
     if (atomicCAS(status, 0u, code) == 0u) status[1] = detail;
 }
@@ -61,7 +92,7 @@ inline int grouped_token_tile(int64_t M, int V) {
     const int64_t avg = M / (V > 0 ? V : 1);
     return avg <= 48 ? 64 : (avg <= 100 ? 128 : 256);
 }
-// The 256-row x 256-token tiles on CTA pairs are in use (PD_GEMM_PAIR=0 turns them off, for comparisons).
+// Layers with at least 256 output rows run on CTA pairs (256-row tiles); smaller ones on one CTA per 128-row tile.
 bool gemm_pair_enabled();
 // Token tile the multi-variant path cuts buckets into: 256 when the pair kernel takes them.
 inline int grouped_token_tile_for(int64_t M, int V, int64_t d_out) {
@@ -72,6 +103,15 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
                               uint32_t *status, cudaStream_t stream);
+
+// Multi-variant decode: at most kMvDecodeMaxTokens token rows, d_in a multiple of 128.  One launch, one pass over
+// W_b; the kernel buckets the rows by variant id itself (ids outside [-1, V) latch PD_ERR_BAD_VARIANT).
+constexpr int kMvDecodeMaxTokens = 64;
+size_t mv_decode_scratch_bytes(int64_t M, int32_t V, int64_t d_in);  // x and col-axis scales in the kernel's own layout
+pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *ids, const __half *w_b, const uint32_t *masks,
+                           int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits, int V,
+                           int64_t d_out, int64_t d_in, __half *y, int64_t ldy, unsigned char *scratch, uint32_t *status,
+                           cudaStream_t stream);
 
 // Stable bucket sort of token rows by variant id: offsets[g] .. offsets[g+1] index row_index for
 // variant g (g = 0..V-1), offsets[V] .. offsets[V+1] the rows with id -1.  Other ids latch an error.

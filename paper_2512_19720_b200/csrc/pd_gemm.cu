@@ -29,8 +29,6 @@
 // warps take the even steps, four the odd ones.
 // Every wait is bounded; a wait that runs out latches PD_ERR_DEVICE_TIMEOUT and the CTA
 // drains and exits.
-#include <cstdlib>
-
 #include "pd_ptx.cuh"
 
 namespace pd {
@@ -850,10 +848,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 // ------------------------------------------------------------------ host side
 }  // namespace
 
-bool gemm_pair_enabled() {
-    static const bool on = [] { const char *e = getenv("PD_GEMM_PAIR"); return e ? atoi(e) != 0 : true; }();
-    return on;
-}
+bool gemm_pair_enabled() { return true; }
 
 namespace {
 // fp16 row-major [rows, cols] with row pitch ld elements; box = 64 columns x box_rows rows, 128-byte swizzle
@@ -866,11 +861,8 @@ template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
 pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
     auto kernel = gemm_kernel<AXIS, HAS_DELTA, GROUPED, BN>;
     constexpr int smem = SmemLayout<BN>::kTotal;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return PD_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
+    if (!ensure_dynamic_smem(kernel, smem, configured)) return PD_ERR_CUDA;
     kernel<<<grid, kNumThreads, smem, stream>>>(mw, mx, args);
     count_launch();
     return cuda_ok(cudaGetLastError());
@@ -914,11 +906,8 @@ template <int AXIS, bool HAS_DELTA, bool GROUPED>
 pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
     auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA, GROUPED>;
     constexpr int smem = PairLayout::kTotal;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return PD_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
+    if (!ensure_dynamic_smem(kernel, smem, configured)) return PD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(pair_threads(GROUPED));
@@ -1005,7 +994,6 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
         // CTA pairs, tiles of 256 rows x token_tile tokens.  A pair of k steps costs the issuing thread about 1250
         // clocks whatever the tile's width (the MMA instruction rate), the tensor cores 4 clocks per token; pick the
         // width with the fewest rounds x that, ties to the narrower tile (more CTAs stream the weights).
-        static const int forced = [] { const char *e = getenv("PD_GEMM_TOKEN_TILE"); return e ? atoi(e) : 0; }();
         const int64_t tiles_m2 = (d_out + 2 * BM - 1) / (2 * BM);
         const int pairs = sms / 2;
         int best_tt = 256;
@@ -1016,7 +1004,6 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
             const int64_t cost = ((units + pairs - 1) / pairs) * per;
             if (best_tt_cost < 0 || cost <= best_tt_cost) best_tt = tt, best_tt_cost = cost;
         }
-        if (forced == 64 || forced == 128 || forced == 256) best_tt = forced;
         return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, best_tt, status, stream);
     }
     // One CTA per tile (fewer than 256 output rows).  256 tokens per tile amortise the W_hat transform best, but with

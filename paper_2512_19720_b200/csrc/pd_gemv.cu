@@ -1,45 +1,11 @@
-// Decode path: y[M<=16, d_out] = x . (W_b + v (.) B)^T, bound by HBM (2.125 bytes per weight).
+// Decode path: y[M<=16, d_out] = x . (W_b + v (.) B)^T, bound by HBM (2.125 bytes per weight element).
 //
-// The product is split as  y = x.W_b^T + s (.) (x'.B^T)  with x' = x (row axis, s = v applied to
-// the output) or x' = x*v (col axis, s = 1), so W_hat is never formed, not even in registers.
-//
-// Work decomposition
-//   - a CTA of 8 warps owns 128 output rows (16 per warp = two n8 tiles) and one slice of d_in;
-//     the CTAs of a thread-block cluster (1..8) own consecutive slices of the same rows and
-//     add their partial sums through distributed shared memory in rank order, so the result
-//     does not depend on scheduling;
-//   - a lane streams 16-byte pieces of its W_b row (four per 128-column step and tile) and the
-//     four mask words of the step, expands its 32 mask bits to +-1.0 fp16 pairs with byte
-//     permutes, and feeds both into warp-level m16n8k16 MMAs whose M dimension is the token
-//     index.  The k order inside a step is permuted the same way for x and for W, so no
-//     shuffle is needed; the k reduction across lanes happens inside the MMA.
-//   - the x slice (and x*v for the col axis) is staged once per CTA in shared memory.
-#include <cooperative_groups.h>
-
-#include <cstdlib>
-
+// gemv_stream_kernel (below) is the product path for every d_in that is a multiple of 128; gemv_generic_kernel
+// (one warp per output row, plain FMAs) covers the remaining shapes and is not tuned.
 #include "pd_ptx.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace pd {
 namespace {
-
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kRowsPerCta = kWarps * 16;
-constexpr int kStepK = 128;       // columns per warp step
-constexpr int kPhaseSteps = 8;    // steps whose x slice is resident in shared memory at once
-constexpr int kPhaseK = kStepK * kPhaseSteps;
-constexpr int kXStride = kPhaseK + 32;  // halves; +64 bytes keeps the 8 token rows on distinct banks
-
-__device__ __forceinline__ uint4 ldg_stream(const void *p) {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
-    return r;
-}
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -49,6 +15,7 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// arguments of the generic kernel
 struct GemvArgs {
     const __half *x;
     const __half *w_b;
@@ -57,185 +24,12 @@ struct GemvArgs {
     __half *y;
     int64_t ldx, ldy;
     int M, d_out, d_in;
-    int steps_total;  // d_in / 128
     // grouped mode (multi-variant): the tokens of this launch are rows
     // row_index[group_offsets[group] .. group_offsets[group + 1]) of x and y; M is ignored
     const int *row_index;
     const int *group_offsets;
     int group;
 };
-
-struct StepRegs {
-    uint4 w[2][4];  // [tile][chunk]: 8 halves of the lane's row at k = step*128 + 32*chunk + 8*t
-    uint4 m[2];     // [tile]: the 4 mask words of the step
-};
-
-template <bool HAS_DELTA>
-__device__ __forceinline__ void load_step(StepRegs &r, const __half *const (&wrow)[2],
-                                          const uint32_t *const (&mrow)[2], int step, int t) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const __half *p = wrow[j] + static_cast<size_t>(step) * kStepK + 8 * t;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) r.w[j][c] = ldg_stream(p + 32 * c);
-        if (HAS_DELTA) r.m[j] = ldg_stream(mrow[j] + 4 * step);
-    }
-}
-
-// AXIS: PD_AXIS_ROW / PD_AXIS_COL.  HAS_DELTA false: base weights only.  M16: more than 8 tokens.
-template <int AXIS, bool HAS_DELTA, bool M16>
-__global__ void __launch_bounds__(kThreads, 2) gemv_kernel(const GemvArgs a) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    constexpr int kTokRows = M16 ? 16 : 8;
-    constexpr bool kScaledCopy = HAS_DELTA && AXIS == PD_AXIS_COL;
-    __half *xs = reinterpret_cast<__half *>(smem);                  // [kTokRows][kXStride]
-    __half *xv = xs + (kScaledCopy ? kTokRows * kXStride : 0);      // x*v copy (col axis)
-    float *part = reinterpret_cast<float *>(smem + (kScaledCopy ? 2 : 1) * kTokRows * kXStride * sizeof(__half));
-    // part: [16][kRowsPerCta] partial sums of this CTA
-
-    cg::cluster_group cluster = cg::this_cluster();
-    const int n_rank = static_cast<int>(cluster.num_blocks());
-    const int rank = static_cast<int>(cluster.block_rank());
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int g = lane >> 2, t = lane & 3;
-    const int row_base = blockIdx.y * kRowsPerCta + warp * 16;
-
-    int n_tok = a.M;
-    const int *tok_rows = nullptr;
-    if (a.group_offsets != nullptr) {
-        const int first = a.group_offsets[a.group];
-        n_tok = a.group_offsets[a.group + 1] - first;
-        tok_rows = a.row_index + first;
-    }
-
-    const int step0 = static_cast<int>((static_cast<int64_t>(rank) * a.steps_total) / n_rank);
-    const int step1 = static_cast<int>((static_cast<int64_t>(rank + 1) * a.steps_total) / n_rank);
-
-    const __half *wrow[2];
-    const uint32_t *mrow[2];
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const int row = min(row_base + 8 * j + g, a.d_out - 1);  // rows past the end re-read the last row
-        wrow[j] = a.w_b + static_cast<size_t>(row) * a.d_in;
-        mrow[j] = HAS_DELTA ? a.mask + static_cast<size_t>(row) * (a.d_in >> 5) : nullptr;
-    }
-
-    const uint32_t sel_pick = static_cast<uint32_t>(t | ((4 + t) << 4));  // byte t of two words
-
-  // chunks of up to 16 (M16) or 8 tokens; a plain call has exactly one chunk
-  for (int tok0 = 0; tok0 < n_tok; tok0 += kTokRows) {
-    const int M = min(kTokRows, n_tok - tok0);
-    float acc_b[2][4], acc_d[2][4];
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc_b[j][i] = acc_d[j][i] = 0.f;
-
-    for (int ph0 = step0; ph0 < step1; ph0 += kPhaseSteps) {
-        const int ph1 = min(ph0 + kPhaseSteps, step1);
-        StepRegs cur;
-        load_step<HAS_DELTA>(cur, wrow, mrow, ph0, t);  // in flight while x is staged
-
-        __syncthreads();  // previous phase's readers are done
-        {
-            const int k0 = ph0 * kStepK, vec_per_row = (ph1 - ph0) * (kStepK / 8);
-            for (int i = threadIdx.x; i < kTokRows * vec_per_row; i += kThreads) {
-                const int m = i / vec_per_row, c = i - m * vec_per_row;
-                uint4 val = make_uint4(0, 0, 0, 0);
-                if (m < M) {
-                    const int xr = tok_rows ? tok_rows[tok0 + m] : tok0 + m;
-                    val = *reinterpret_cast<const uint4 *>(a.x + static_cast<size_t>(xr) * a.ldx + k0 + 8 * c);
-                }
-                *reinterpret_cast<uint4 *>(xs + m * kXStride + 8 * c) = val;
-                if (kScaledCopy) {
-                    const uint4 vv = *reinterpret_cast<const uint4 *>(a.v + k0 + 8 * c);
-                    uint4 sc;
-                    const __half2 *xp = reinterpret_cast<const __half2 *>(&val);
-                    const __half2 *vp = reinterpret_cast<const __half2 *>(&vv);
-                    __half2 *sp = reinterpret_cast<__half2 *>(&sc);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) sp[q] = __hmul2(xp[q], vp[q]);
-                    *reinterpret_cast<uint4 *>(xv + m * kXStride + 8 * c) = sc;
-                }
-            }
-        }
-        __syncthreads();
-
-        for (int step = ph0; step < ph1; ++step) {
-            StepRegs nxt;
-            if (step + 1 < ph1) load_step<HAS_DELTA>(nxt, wrow, mrow, step + 1, t);
-            const int kk = (step - ph0) * kStepK + 8 * t;
-
-            uint32_t sh[2][8];
-            if (HAS_DELTA) {
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const uint32_t lo = prmt(cur.m[j].x, cur.m[j].y, sel_pick);
-                    const uint32_t hi = prmt(cur.m[j].z, cur.m[j].w, sel_pick);
-                    const uint32_t my = prmt(lo, hi, 0x5410u);  // byte c = this lane's 8 bits of chunk c
-#pragma unroll
-                    for (int s = 0; s < 8; ++s) sh[j][s] = my << s;  // bit 8c+q sits on top of byte c in sh[7-q]
-                }
-            }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint4 xa = *reinterpret_cast<const uint4 *>(xs + g * kXStride + kk + 32 * c);
-                uint4 xb = make_uint4(0, 0, 0, 0);
-                if (M16) xb = *reinterpret_cast<const uint4 *>(xs + (g + 8) * kXStride + kk + 32 * c);
-                uint4 da = xa, db = xb;
-                if (kScaledCopy) {
-                    da = *reinterpret_cast<const uint4 *>(xv + g * kXStride + kk + 32 * c);
-                    if (M16) db = *reinterpret_cast<const uint4 *>(xv + (g + 8) * kXStride + kk + 32 * c);
-                }
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const uint4 w = cur.w[j][c];
-                    mma16816(acc_b[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                    mma16816(acc_b[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
-                    if (HAS_DELTA) {
-                        // pair r holds the signs of halves 2r (low) and 2r+1 (high) of chunk c
-                        const uint32_t sel = static_cast<uint32_t>(((c | 8) << 4) | (((4 + c) | 8) << 12));
-                        uint32_t pm[4];
-#pragma unroll
-                        for (int r = 0; r < 4; ++r)
-                            pm[r] = lop3_andn_or(prmt(sh[j][7 - 2 * r], sh[j][6 - 2 * r], sel), 0x80008000u, 0x3C003C00u);
-                        mma16816(acc_d[j], da.x, db.x, da.y, db.y, pm[0], pm[1]);
-                        mma16816(acc_d[j], da.z, db.z, da.w, db.w, pm[2], pm[3]);
-                    }
-                }
-            }
-            if (step + 1 < ph1) cur = nxt;
-        }
-    }
-
-    // this CTA's partial sums -> shared memory, [token][row in CTA]
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int ol = warp * 16 + 8 * j + 2 * t + e;
-            float s = 1.f;
-            if (HAS_DELTA && AXIS == PD_AXIS_ROW) s = __half2float(a.v[min(blockIdx.y * kRowsPerCta + ol, a.d_out - 1)]);
-            part[g * kRowsPerCta + ol] = acc_b[j][e] + (HAS_DELTA ? s * acc_d[j][e] : 0.f);
-            if (M16) part[(g + 8) * kRowsPerCta + ol] = acc_b[j][2 + e] + (HAS_DELTA ? s * acc_d[j][2 + e] : 0.f);
-        }
-    }
-    cluster.sync();
-    {
-        // rank r adds up rows [r*seg, (r+1)*seg) of every token, over the ranks in order
-        const int seg = kRowsPerCta / n_rank;
-        for (int i = threadIdx.x; i < M * seg; i += kThreads) {
-            const int m = i / seg, ol = rank * seg + (i - m * seg);
-            float sum = 0.f;
-            for (int q = 0; q < n_rank; ++q) sum += cluster.map_shared_rank(part, q)[m * kRowsPerCta + ol];
-            const int o = blockIdx.y * kRowsPerCta + ol;
-            const int yr = tok_rows ? tok_rows[tok0 + m] : tok0 + m;
-            if (o < a.d_out) a.y[static_cast<size_t>(yr) * a.ldy + o] = __float2half_rn(sum);
-        }
-    }
-    cluster.sync();  // keep shared memory alive until every rank has read it
-  }
-}
 
 // ---------------------------------------------------------------------------------------------
 // Streaming decode kernel: weights brought in by TMA, one CTA per 16 output rows, two or three CTAs per SM.
@@ -585,51 +379,13 @@ __global__ void __launch_bounds__(256) gemv_generic_kernel(const GemvArgs a) {
   }
 }
 
-int env_int(const char *name, int fallback) {
-    const char *s = getenv(name);
-    return s ? atoi(s) : fallback;
-}
-
-template <int AXIS, bool HAS_DELTA, bool M16>
-pd_status launch_variant(const GemvArgs &args, int n_rank, cudaStream_t stream) {
-    constexpr int tok = M16 ? 16 : 8;
-    constexpr bool scaled = HAS_DELTA && AXIS == PD_AXIS_COL;
-    const size_t smem = static_cast<size_t>(scaled ? 2 : 1) * tok * kXStride * sizeof(__half) +
-                        16 * kRowsPerCta * sizeof(float);
-    auto kernel = gemv_kernel<AXIS, HAS_DELTA, M16>;
-    static bool configured = false;  // per instantiation
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-            return PD_ERR_CUDA;
-        configured = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(n_rank), static_cast<unsigned>((args.d_out + kRowsPerCta - 1) / kRowsPerCta));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(n_rank);
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    count_launch();
-    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, args));
-}
-
 template <int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
 pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, const StreamArgs &args, int grid,
                                 cudaStream_t stream) {
     auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16, KS, STAGES>;
     constexpr int kStreamSmem = stream_smem_bytes(KS, STAGES);
-    static bool configured = false;  // per instantiation
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem) != cudaSuccess)
-            return PD_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
+    if (!ensure_dynamic_smem(kernel, kStreamSmem, configured)) return PD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(kStreamThreads);
@@ -639,8 +395,7 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, co
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may start while the previous kernel drains
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const int use_pdl = env_int("PD_PDL", 1);
-    cfg.numAttrs = use_pdl ? 1 : 0;
+    cfg.numAttrs = 1;
     count_launch();
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mm, args));
 }
@@ -692,10 +447,9 @@ pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, 
     // wave is not much emptier than with two CTAs per SM.  Measured and dropped: tiles of 32 rows (half the x
     // traffic, but too few consumer warps per SM on small grids) and tiles of 12-15 rows (fill every SM when
     // d_out / 16 is just under a wave, but the consumers' work per CTA does not shrink with the tile).
-    static const int forced = env_int("PD_GEMV_CTAS_PER_SM", 0);  // 2 or 3; 0 = by the rule below
     const double tiles = static_cast<double>((d_out + kStreamRows - 1) / kStreamRows);
     const double w3 = tiles / (3.0 * sm_count()), w2 = tiles / (2.0 * sm_count());
-    const bool three = forced ? forced == 3 : (w3 >= 1.0 && w3 / ceil(w3) >= w2 / ceil(w2) - 0.1);
+    const bool three = w3 >= 1.0 && w3 / ceil(w3) >= w2 / ceil(w2) - 0.1;
     if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
     return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
 }
@@ -707,8 +461,7 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       const int *row_index, const int *group_offsets, int group, const GemvScratch *ws,
                       cudaStream_t stream) {
     // plain calls on TMA-friendly shapes stream the weights through shared memory
-    static const int use_stream = env_int("PD_GEMV_STREAM", 1);
-    if (use_stream && ws != nullptr && group_offsets == nullptr && d_in % 128 == 0)
+    if (ws != nullptr && group_offsets == nullptr && d_in % 128 == 0)
         return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, stream);
     GemvArgs args;
     args.x = x;
@@ -721,45 +474,17 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
     args.M = M;
     args.d_out = static_cast<int>(d_out);
     args.d_in = static_cast<int>(d_in);
-    args.steps_total = static_cast<int>(d_in / kStepK);
     args.row_index = row_index;
     args.group_offsets = group_offsets;
     args.group = group;
-    if (d_in % kStepK != 0) {
-        const int rows_per_cta = 8;
-        const unsigned grid = static_cast<unsigned>((d_out + rows_per_cta - 1) / rows_per_cta);
-        if (axis == PD_AXIS_ROW)
-            gemv_generic_kernel<PD_AXIS_ROW><<<grid, 256, 0, stream>>>(args);
-        else
-            gemv_generic_kernel<PD_AXIS_COL><<<grid, 256, 0, stream>>>(args);
-        count_launch();
-        return cuda_ok(cudaGetLastError());
-    }
-    // k split: as many cluster ranks (<= 8, power of two) as keep at least 2 steps per rank and
-    // are needed to put about two CTAs on every SM
-    static const int forced = env_int("PD_GEMV_CLUSTER", 0);
-    int n_rank = 8;
-    if (forced == 1 || forced == 2 || forced == 4 || forced == 8) {
-        n_rank = forced;
-    } else {
-        const int64_t row_blocks = (d_out + kRowsPerCta - 1) / kRowsPerCta;
-        while (n_rank > 1 && (args.steps_total / n_rank < 2 || row_blocks * (n_rank / 2) >= 2 * 148)) n_rank >>= 1;
-    }
-    while (n_rank > 1 && args.steps_total < n_rank) n_rank >>= 1;
-    const bool m16 = M > 8 || group_offsets != nullptr;
-    const bool delta = mask != nullptr;
-#define PD_GEMV_CASE(AX, D, W) return launch_variant<AX, D, W>(args, n_rank, stream)
-    if (!delta) {
-        if (m16) PD_GEMV_CASE(PD_AXIS_ROW, false, true);
-        PD_GEMV_CASE(PD_AXIS_ROW, false, false);
-    }
-    if (axis == PD_AXIS_ROW) {
-        if (m16) PD_GEMV_CASE(PD_AXIS_ROW, true, true);
-        PD_GEMV_CASE(PD_AXIS_ROW, true, false);
-    }
-    if (m16) PD_GEMV_CASE(PD_AXIS_COL, true, true);
-    PD_GEMV_CASE(PD_AXIS_COL, true, false);
-#undef PD_GEMV_CASE
+    const int rows_per_cta = 8;
+    const unsigned grid = static_cast<unsigned>((d_out + rows_per_cta - 1) / rows_per_cta);
+    if (axis == PD_AXIS_ROW)
+        gemv_generic_kernel<PD_AXIS_ROW><<<grid, 256, 0, stream>>>(args);
+    else
+        gemv_generic_kernel<PD_AXIS_COL><<<grid, 256, 0, stream>>>(args);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
 }
 
 }  // namespace pd

@@ -308,7 +308,6 @@ namespace {
 constexpr int64_t kStaticSumWords = 65536;  // d_out + d_in may not exceed this
 static __device__ __align__(256) unsigned long long g_static_sums[kStaticSumWords];
 
-constexpr int kMaxDevices = 64;
 std::atomic<unsigned long long *> g_static_sums_addr[kMaxDevices];
 
 // Device address of g_static_sums on the current device (nullptr on failure).
