@@ -20,6 +20,9 @@
  *     pd_workspace_bytes() tells how much a call needs.  The workspace must be 256-byte aligned,
  *     and its first 256 bytes (the device status words) must be zero when it is first handed to
  *     the library: zero-fill it once after allocating it.  pd_device_status() re-zeroes them.
+ *     pd_pack_delta needs ALL of its workspace zero on entry and leaves all of it zero on return
+ *     (see there); the linear calls overwrite theirs beyond the status words, so give
+ *     pd_pack_delta a workspace of its own or zero-fill it again after another call has used it.
  *   - cuda_stream is a cudaStream_t passed as void* (NULL = the legacy default stream).  Every
  *     call only enqueues work on that stream and returns without synchronising.
  *   - Errors that can be seen on the host (NULL pointers, bad sizes, misalignment, a short
@@ -75,7 +78,11 @@ typedef enum {
  *
  * The sums of |dW| are accumulated exactly (fixed point, units of 2^-24), divided once in fp64
  * and rounded once to fp16, so the result does not depend on launch shape or summation order.
- * Non-finite inputs are outside the contract.  Needs pd_workspace_bytes(PD_OP_PACK, ...).
+ * Non-finite inputs are outside the contract.
+ * Workspace: pd_workspace_bytes(PD_OP_PACK, ...) bytes that are ALL ZERO when the call is made (zero-fill once
+ * after allocation); the sums are added into it and the call puts every byte back to zero before it completes,
+ * so calls queued one after another on a stream can share it.  Calls that overlap on the GPU need workspaces of
+ * their own.
  */
 pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in,
                         uint32_t *mask, void *v_row, void *v_col,
@@ -104,17 +111,34 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx,
                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * pd_linear_ex -- pd_linear with flags (same operation, same paper passages).
+ *
+ *   PD_LINEAR_WEIGHTS_RESIDENT : the caller vouches that w_b, mask and v are not written by any work queued earlier
+ *       on cuda_stream that may still be running (the serving case: weights loaded once, then many calls).  The
+ *       decode kernel (M <= 16) is launched so that it can start while the previous kernel on the stream drains;
+ *       with this flag it streams the weights at once and only x and y wait for that kernel.  Without the flag
+ *       (pd_linear) every load waits, so pd_pack_delta -> pd_linear and pd_merge -> pd_linear(w_hat, mask = NULL)
+ *       back to back on one stream are always correct.  The flag has no effect for M > 16.
+ */
+#define PD_LINEAR_WEIGHTS_RESIDENT 1u
+pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx,
+                       const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
+                       int64_t d_out, int64_t d_in, void *y, int64_t ldy,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream, uint32_t flags);
+
+/*
  * pd_linear_host -- pd_linear for activations that live in HOST memory (same operation and paper passages
  * as pd_linear).  Enqueues, on cuda_stream: copy of x_host -> x_dev, the fused linear, copy of y_dev -> y_host.
  *
  *   x_host : in,  HOST fp16 [M, d_in], dense (row stride d_in); pinned memory makes the copies asynchronous
  *   y_host : out, HOST fp16 [M, d_out], dense
  *   x_dev, y_dev : device staging buffers owned by the caller, at least M*d_in and M*d_out fp16, 16-byte aligned
+ *   flags  : as in pd_linear_ex (0 or PD_LINEAR_WEIGHTS_RESIDENT)
  *   everything else as in pd_linear.  The results are in y_host once the stream has been synchronised.
  */
 pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void *w_b, const uint32_t *mask,
                          const void *v, pd_axis axis, int64_t d_out, int64_t d_in, void *y_dev, void *y_host,
-                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+                         void *workspace, size_t workspace_bytes, void *cuda_stream, uint32_t flags);
 
 /*
  * pd_linear_multivariant -- one batch, many fine-tunes over one base.
@@ -128,7 +152,10 @@ pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void 
  *   vs          : in, fp16 [V, v_stride]; variant g's scales start at vs + g*v_stride
  *   axes        : in, HOST array of V bytes, each a pd_axis
  *
- * Everything else as in pd_linear.  V <= 64.
+ * Everything else as in pd_linear, except that a batch of at most 64 rows (d_in a multiple of 128) keeps the
+ * products x.W_b and x.(+-v) apart in exact fp16 x fp16 products (W_hat is not rounded to fp16 first).  V <= 64.
+ * Batches of at most 64 rows run as one pass over W_b: HBM traffic is W_b plus the masks of the variants present.
+ * Needs pd_workspace_bytes(PD_OP_LINEAR_MULTIVARIANT, M, V, ...).
  */
 pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids,
                                  const void *w_b, const uint32_t *masks, const void *vs,
@@ -165,9 +192,9 @@ pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis
  *   set-up    : the first call on each device looks up the array's device address (the device
  *               must be current, as for every call).  Make that first call outside any stream
  *               capture.
- *   sharing   : all calls on one GPU use the same array.  Each call zero-fills the part it uses
- *               on its stream first, so back-to-back calls on ONE stream are safe; calls that may
- *               overlap on the GPU (different streams, different threads) race on it and give
+ *   sharing   : all calls on one GPU use the same array.  It starts zero-filled and each call puts
+ *               what it used back to zero, so back-to-back calls on ONE stream are safe; calls that
+ *               may overlap on the GPU (different streams, different threads) race on it and give
  *               wrong scales -- serialise them or use pd_pack_delta with separate workspaces.
  *   It calls no cudaMalloc / cudaFree and no allocating library routine.
  */
@@ -181,6 +208,16 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
 /* Synchronises the stream, reads the status word that the last pd_linear* call on this
  * workspace latched, clears it and returns it (PD_OK when nothing was latched). */
 pd_status pd_device_status(void *workspace, void *cuda_stream);
+
+/*
+ * pd_selftest_bounded_wait -- exercises the device-side failure path without a fault.
+ * Every wait inside the kernels (on a TMA copy, on another warp, on the other CTA of a pair) is bounded: when it
+ * runs out the kernel latches PD_ERR_DEVICE_TIMEOUT in the workspace status words and returns.  This call launches
+ * one warp that waits, with that same routine and a limit of limit_cycles SM clocks (1 .. 1e8), on a barrier that
+ * nothing arrives on; afterwards pd_device_status(workspace) returns PD_ERR_DEVICE_TIMEOUT once, then PD_OK.
+ * The GPU context stays usable.  workspace: at least 256 bytes, 256-byte aligned, zero-filled.
+ */
+pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream);
 
 /* Human-readable name of a status code; never NULL. */
 const char *pd_status_string(pd_status status);

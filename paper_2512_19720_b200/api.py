@@ -18,8 +18,9 @@ OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE = 0, 1, 2, 3
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpd.so")
 
-EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_multivariant", "pd_merge", "pd_workspace_bytes",
-           "pd_device_status", "pd_status_string", "pd_launch_count"]
+EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_ex", "pd_linear_multivariant", "pd_merge",
+           "pd_workspace_bytes", "pd_device_status", "pd_status_string", "pd_launch_count", "pd_selftest_bounded_wait"]
+LINEAR_WEIGHTS_RESIDENT = 1
 
 
 class PdError(RuntimeError):
@@ -40,8 +41,12 @@ def _load() -> ctypes.CDLL:
     lib.pd_pack_delta_static.restype = ctypes.c_int
     lib.pd_linear.argtypes = [p, i64, i64, p, p, p, ctypes.c_int, i64, i64, p, i64, p, sz, p]
     lib.pd_linear.restype = ctypes.c_int
-    lib.pd_linear_host.argtypes = [p, p, i64, p, p, p, ctypes.c_int, i64, i64, p, p, p, sz, p]
+    lib.pd_linear_ex.argtypes = [p, i64, i64, p, p, p, ctypes.c_int, i64, i64, p, i64, p, sz, p, ctypes.c_uint32]
+    lib.pd_linear_ex.restype = ctypes.c_int
+    lib.pd_linear_host.argtypes = [p, p, i64, p, p, p, ctypes.c_int, i64, i64, p, p, p, sz, p, ctypes.c_uint32]
     lib.pd_linear_host.restype = ctypes.c_int
+    lib.pd_selftest_bounded_wait.argtypes = [p, i64, p]
+    lib.pd_selftest_bounded_wait.restype = ctypes.c_int
     lib.pd_linear_multivariant.argtypes = [p, i64, i64, p, p, p, p, i64, p, i32, i64, i64, p, i64, p, sz, p]
     lib.pd_linear_multivariant.restype = ctypes.c_int
     lib.pd_merge.argtypes = [p, p, p, ctypes.c_int, i64, i64, p, p]
@@ -85,6 +90,20 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
     return ws
 
 
+_pack_ws_cache: dict = {}
+
+
+def _pack_workspace(nbytes: int, device) -> torch.Tensor:
+    """The pack call's own scratch tensor: it must be all zero on entry, and the call leaves it all zero, so it is
+    kept apart from the workspace the linear calls write into."""
+    key = (device.type, device.index)
+    ws = _pack_ws_cache.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.zeros(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _pack_ws_cache[key] = ws
+    return ws
+
+
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
@@ -104,7 +123,8 @@ def _want(t, dtype, name):
 
 
 def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None, v_col=None, workspace=None):
-    """mask uint32-as-int32 [d_out, d_in/32], v_row fp16 [d_out] | None, v_col fp16 [d_in] | None."""
+    """mask uint32-as-int32 [d_out, d_in/32], v_row fp16 [d_out] | None, v_col fp16 [d_in] | None.
+    A workspace passed in must be all zero (the call leaves it so)."""
     _want(w_f, torch.float16, "w_f"), _want(w_b, torch.float16, "w_b")
     assert w_f.shape == w_b.shape and w_f.is_contiguous() and w_b.is_contiguous()
     d_out, d_in = w_b.shape
@@ -116,7 +136,7 @@ def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None,
     if want_col and v_col is None:
         v_col = torch.empty(d_in, dtype=torch.float16, device=dev)
     need = workspace_bytes(OP_PACK, 0, 0, d_out, d_in)
-    ws = workspace if workspace is not None else _workspace(need, dev)
+    ws = workspace if workspace is not None else _pack_workspace(need, dev)
     _check(lib.pd_pack_delta(_ptr(w_f), _ptr(w_b), d_out, d_in, _ptr(mask), _ptr(v_row if want_row else None),
                              _ptr(v_col if want_col else None), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "pd_pack_delta")
@@ -136,8 +156,9 @@ def pd_pack_delta_static(w_f, w_b, mask, v_row=None, v_col=None):
     return mask, v_row, v_col
 
 
-def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None):
-    """y fp16 [M, d_out] = x . (W_b + v (.) B)^T; mask None = base weights only."""
+def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None, weights_resident=False):
+    """y fp16 [M, d_out] = x . (W_b + v (.) B)^T; mask None = base weights only.  weights_resident=True passes
+    PD_LINEAR_WEIGHTS_RESIDENT: no earlier work on the stream writes w_b, mask or v."""
     _want(x, torch.float16, "x"), _want(w_b, torch.float16, "w_b")
     assert x.dim() == 2 and x.stride(1) == 1 and w_b.is_contiguous()
     m, d_in = x.shape
@@ -147,12 +168,13 @@ def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None):
         y = torch.empty((m, d_out), dtype=torch.float16, device=x.device)
     need = workspace_bytes(OP_LINEAR, m, 0, d_out, d_in)
     ws = workspace if workspace is not None else _workspace(need, x.device)
-    _check(lib.pd_linear(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
-                         y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pd_linear")
+    _check(lib.pd_linear_ex(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
+                            y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
+                            LINEAR_WEIGHTS_RESIDENT if weights_resident else 0), "pd_linear")
     return y
 
 
-def pd_linear_host(x_host, x_dev, w_b, mask, v, axis, y_dev, y_host, workspace=None):
+def pd_linear_host(x_host, x_dev, w_b, mask, v, axis, y_dev, y_host, workspace=None, weights_resident=False):
     """pd_linear with the activations in host memory: x_host (CPU fp16 [M, d_in], ideally pinned) is copied to the
     staging tensor x_dev, the linear runs, y_dev is copied to y_host; all on the current stream, nothing synchronised."""
     assert x_host.dtype == torch.float16 and y_host.dtype == torch.float16 and not x_host.is_cuda and not y_host.is_cuda
@@ -163,8 +185,8 @@ def pd_linear_host(x_host, x_dev, w_b, mask, v, axis, y_dev, y_host, workspace=N
     need = workspace_bytes(OP_LINEAR, m, 0, d_out, d_in)
     ws = workspace if workspace is not None else _workspace(need, w_b.device)
     _check(lib.pd_linear_host(x_host.data_ptr(), _ptr(x_dev), m, _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in,
-                              _ptr(y_dev), y_host.data_ptr(), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
-           "pd_linear_host")
+                              _ptr(y_dev), y_host.data_ptr(), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
+                              LINEAR_WEIGHTS_RESIDENT if weights_resident else 0), "pd_linear_host")
     return y_host
 
 
@@ -196,6 +218,12 @@ def pd_merge(w_b, mask, v, axis, w_hat=None):
         w_hat = torch.empty_like(w_b)
     _check(lib.pd_merge(_ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(w_hat), _stream()), "pd_merge")
     return w_hat
+
+
+def pd_selftest_bounded_wait(limit_cycles=100000, workspace=None, device=None):
+    """Launches the probe whose bounded wait runs out after limit_cycles; pd_device_status() then reports 7 once."""
+    ws = workspace if workspace is not None else _workspace(256, device or torch.device("cuda", torch.cuda.current_device()))
+    _check(lib.pd_selftest_bounded_wait(_ptr(ws), int(limit_cycles), _stream()), "pd_selftest_bounded_wait")
 
 
 def pd_device_status(workspace=None, device=None) -> int:

@@ -2,7 +2,7 @@
 // allocated here; everything runs on the caller's stream.
 #include <climits>
 
-#include "pd_common.cuh"
+#include "pd_ptx.cuh"
 
 namespace pd {
 size_t grouped_table_bytes(int64_t M, int32_t V);
@@ -103,6 +103,20 @@ gather_rows_kernel(const __half *__restrict__ x, int64_t ldx, const int *__restr
     }
 }
 
+// One warp waits, with the library's bounded wait, on an mbarrier that nothing ever arrives on.  The wait gives up
+// after limit_cycles, latches PD_ERR_DEVICE_TIMEOUT (detail 99) and the kernel returns normally.
+__global__ void bounded_wait_probe_kernel(uint32_t *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0, &abort_flag, status, 99, limit_cycles);
+}
+
 pd_status check_matrix_args(const void *x, int64_t M, int64_t ldx, const void *w_b, int64_t d_out, int64_t d_in,
                             const void *y, int64_t ldy) {
     if (!x || !w_b || !y || M <= 0 || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
@@ -145,7 +159,7 @@ extern "C" {
 size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d_in) {
     switch (op) {
         case PD_OP_PACK:
-            return kStatusBytes + round_up(sizeof(unsigned long long) * static_cast<size_t>(d_out + d_in), 256);
+            return kStatusBytes + pack_scratch_bytes(d_out, d_in);
         case PD_OP_LINEAR:
             return kStatusBytes;
         case PD_OP_LINEAR_MULTIVARIANT:
@@ -203,8 +217,15 @@ pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis
 pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
                     pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
                     size_t workspace_bytes, void *cuda_stream) {
+    return pd_linear_ex(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, workspace, workspace_bytes, cuda_stream, 0u);
+}
+
+pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                       pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
     pd_status st = check_matrix_args(x, M, ldx, w_b, d_out, d_in, y, ldy);
     if (st != PD_OK) return st;
+    if (flags & ~static_cast<uint32_t>(PD_LINEAR_WEIGHTS_RESIDENT)) return PD_ERR_INVALID_ARG;
     if (axis != PD_AXIS_ROW && axis != PD_AXIS_COL) return PD_ERR_INVALID_ARG;
     if (mask && !v) return PD_ERR_INVALID_ARG;
     if (mask && (!aligned16(mask) || !aligned16(v))) return PD_ERR_ALIGNMENT;
@@ -218,6 +239,7 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
                            d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), stream);
     GemvScratch scratch;
     scratch.status = static_cast<uint32_t *>(workspace);
+    scratch.weights_resident = (flags & PD_LINEAR_WEIGHTS_RESIDENT) != 0;
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
         const int rows = static_cast<int>(M - m0 < 16 ? M - m0 : 16);
         st = launch_gemv(xh + m0 * ldx, rows, ldx, static_cast<const __half *>(w_b), mask,
@@ -230,13 +252,13 @@ pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, cons
 
 pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void *w_b, const uint32_t *mask, const void *v,
                          pd_axis axis, int64_t d_out, int64_t d_in, void *y_dev, void *y_host, void *workspace,
-                         size_t workspace_bytes, void *cuda_stream) {
+                         size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
     if (!x_host || !x_dev || !y_dev || !y_host || M <= 0 || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * d_in * sizeof(__half), cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return PD_ERR_CUDA;
-    const pd_status st = pd_linear(x_dev, M, d_in, w_b, mask, v, axis, d_out, d_in, y_dev, d_out, workspace, workspace_bytes,
-                                   cuda_stream);
+    const pd_status st = pd_linear_ex(x_dev, M, d_in, w_b, mask, v, axis, d_out, d_in, y_dev, d_out, workspace, workspace_bytes,
+                                      cuda_stream, flags);
     if (st != PD_OK) return st;
     return cuda_ok(cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * d_out * sizeof(__half), cudaMemcpyDeviceToHost, stream));
 }
@@ -297,6 +319,13 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
         if (st != PD_OK) return st;
     }
     return PD_OK;
+}
+
+pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream) {
+    if (!workspace || !aligned256(workspace) || limit_cycles <= 0 || limit_cycles > 100000000) return PD_ERR_INVALID_ARG;
+    bounded_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<uint32_t *>(workspace), limit_cycles);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
 }
 
 pd_status pd_device_status(void *workspace, void *cuda_stream) {

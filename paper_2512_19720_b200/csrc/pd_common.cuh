@@ -61,6 +61,7 @@ __device__ __forceinline__ void latch_error(uint32_t *status, uint32_t code, uin
 }
 
 // --- launchers implemented in the .cu files (all enqueue on `stream`, none synchronises) ---
+size_t pack_scratch_bytes(int64_t d_out, int64_t d_in);  // the sums; zero on entry, zero again on return
 pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
                       __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream);
 pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
@@ -68,7 +69,8 @@ pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v,
 
 // What the decode kernels need from the caller's workspace.
 struct GemvScratch {
-    uint32_t *status;  // device status words
+    uint32_t *status;        // device status words
+    bool weights_resident;   // PD_LINEAR_WEIGHTS_RESIDENT: the weight stream may start before the previous kernel has finished
 };
 
 // M <= 16 tokens (mask == nullptr: base weights only).  With group_offsets != nullptr the tokens are

@@ -57,9 +57,10 @@ struct GemvArgs {
 // as the merge and the prefill path form it) and multiplied with fp32 accumulation.  The eight warps' partial
 // sums are added in warp order through shared memory.
 //
-// Programmatic dependent launch: W_b, mask and v do not depend on the previous kernel in the stream,
-// so the producer starts loading at once; the consumers wait for the previous kernel
-// (griddepcontrol.wait) before they touch x or y.
+// Programmatic dependent launch: the kernel may start while the previous kernel in the stream drains.  The
+// consumers wait for that kernel (griddepcontrol.wait) before they touch x or y; the producer waits too, unless
+// the caller has declared the weights resident (PD_LINEAR_WEIGHTS_RESIDENT), in which case it streams W_b, mask
+// and v at once.
 constexpr int kStreamConsumers = 8;
 constexpr int kStreamThreads = (kStreamConsumers + 1) * 32;
 constexpr int kStreamRows = 16;             // output rows per CTA
@@ -83,6 +84,7 @@ struct StreamArgs {
     int64_t ldx, ldy;
     int M, d_out, d_in;
     int n_k;      // steps of KS columns (the last one may be partly past d_in)
+    int weights_resident;  // W_b, mask and v are not written by earlier work on the stream: load them before the grid dependency resolves
     uint32_t *status;
 };
 
@@ -147,6 +149,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // ------------------------------------------------ producer
         if (lane == 0) {
             grid_launch_dependents();  // the next kernel in the stream may start its own weight loads
+            // Unless the caller vouches that no earlier work on the stream writes the weights, they may be the
+            // previous kernel's output (pd_pack_delta or pd_merge right before this call): wait for it like the consumers.
+            if (!a.weights_resident) grid_dependency_wait();
             uint32_t gs = 0;           // steps issued so far
             bool ok = true;
             {
@@ -403,7 +408,7 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, co
 template <int KS, int STAGES>
 pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                              int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                             cudaStream_t stream) {
+                             bool weights_resident, cudaStream_t stream) {
     constexpr int step = KS, R = kStreamRows;
     const bool m16 = M > 8, delta = mask != nullptr;
     CUtensorMap mw, mm;
@@ -420,6 +425,7 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
     a.d_out = static_cast<int>(d_out);
     a.d_in = static_cast<int>(d_in);
     a.n_k = static_cast<int>((d_in + step - 1) / step);
+    a.weights_resident = weights_resident ? 1 : 0;
     a.status = status;
     // one CTA per tile of R rows: a persistent grid walking several tiles measured slower on the 7B
     // shapes (fewer rings in flight, more registers)
@@ -440,7 +446,7 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
 
 pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                         int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                        cudaStream_t stream) {
+                        bool weights_resident, cudaStream_t stream) {
     // Ring depth.  A shorter ring (four steps, 72 KB) lets three CTAs share an SM: the same bytes in flight,
     // but a CTA that is finishing (last step, reduction, store) overlaps two that stream.  It needs a grid that
     // fills three CTAs per SM (smaller grids need six steps per CTA to keep enough in flight) and whose last
@@ -450,8 +456,8 @@ pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, 
     const double tiles = static_cast<double>((d_out + kStreamRows - 1) / kStreamRows);
     const double w3 = tiles / (3.0 * sm_count()), w2 = tiles / (2.0 * sm_count());
     const bool three = w3 >= 1.0 && w3 / ceil(w3) >= w2 / ceil(w2) - 0.1;
-    if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
-    return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, stream);
+    return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, stream);
 }
 
 }  // namespace
@@ -462,7 +468,7 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       cudaStream_t stream) {
     // plain calls on TMA-friendly shapes stream the weights through shared memory
     if (ws != nullptr && group_offsets == nullptr && d_in % 128 == 0)
-        return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, stream);
+        return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, ws->weights_resident, stream);
     GemvArgs args;
     args.x = x;
     args.w_b = w_b;

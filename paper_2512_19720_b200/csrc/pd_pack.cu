@@ -1,10 +1,12 @@
-// pack: sign mask of W_f - W_b plus the exact per-axis sums of |W_f - W_b|, and
+// pack: sign mask of W_f - W_b plus the exact per-axis means of |W_f - W_b|, and
 // merge: W_hat = fp16(fp32(W_b) +- fp32(v)).  Both are single-pass streaming kernels bound by HBM
 // (4.125 bytes per weight element each).
 //
-// Tile shape for both: a CTA of 8 warps covers 64 rows x 256 columns; a warp owns one row at a
+// Tile shape: a CTA of 8 warps covers 32 (pack) or 64 (merge) rows x 256 columns; a warp owns one row at a
 // time, a lane owns 8 consecutive columns (one 128-bit load per matrix), so four neighbouring
 // lanes form one 32-bit mask word.
+#include <climits>
+
 #include "pd_common.cuh"
 
 namespace pd {
@@ -14,7 +16,8 @@ std::atomic<int64_t> g_launches{0};
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kTileRows = 64;
+constexpr int kTileRows = 64;   // merge
+constexpr int kPackRows = 32;   // pack
 constexpr int kTileCols = 256;
 constexpr unsigned kFull = 0xffffffffu;
 
@@ -51,145 +54,177 @@ __device__ __forceinline__ long long half_units(uint32_t h) {
     return (h & 0x8000u) ? -mag : mag;
 }
 
-// |a - b| in units of 2^-24 for two binary16 values less than 0.5 apart: the fp32 difference is exact
-// (a multiple of 2^-24 below 2^23 units), and adding 0.5 places it where one fp32 ulp is 2^-24.  For
-// values 0.5 or more apart the result is >= 2^23 (or has high bits set), which the caller tests.
-__device__ __forceinline__ uint32_t abs_diff_units_small(float a, float b) {
-    return __float_as_uint(fabsf(__fsub_rn(a, b)) + 0.5f) - 0x3f000000u;
+// mean = (sum * 2^-24) / n with one fp64 division, then one rounding to binary16
+__device__ __forceinline__ unsigned short mean_to_half(unsigned long long sum, int n) {
+    const double q = __ddiv_rn(static_cast<double>(sum), static_cast<double>(n)) * 5.9604644775390625e-08;  // 2^-24, exact scaling
+    unsigned short h;
+    asm("cvt.rn.f16.f64 %0, %1;" : "=h"(h) : "d"(q));
+    return h;
 }
 
-// Programmatic dependent launch: a pack call is three kernels (zero the sums, pack, finalize).  Each lets the
-// next one be scheduled as soon as it has started and the next one waits for it before it touches the sums, so
-// the launch latencies overlap the kernels instead of adding to them.
+// One row of a tile, any position: bounds-checked, exact 64-bit fixed point for every magnitude.  Used for tiles that
+// hang over the matrix edge and for the rare tiles that hold a |dW| >= 0.5.
+template <bool ROW, bool COL>
+__device__ __forceinline__ void pack_row_exact(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int o, int col0,
+                                               int d_out, int d_in, uint32_t *__restrict__ mask,
+                                               unsigned long long *__restrict__ row_sum,
+                                               unsigned long long *__restrict__ col_sum, int lane) {
+    const bool ok = o < d_out && col0 < d_in;
+    uint32_t bits = 0;
+    unsigned long long sum = 0;
+    if (ok) {
+        const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
+        const uint4 a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
+        const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p]));
+            bits |= ((ge & 1u) << (2 * p)) | (((ge >> 16) & 1u) << (2 * p + 1));
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const long long d = half_units((a[p] >> (16 * h)) & 0xffffu) - half_units((b[p] >> (16 * h)) & 0xffffu);
+                const unsigned long long du = static_cast<unsigned long long>(d < 0 ? -d : d);
+                sum += du;
+                if (COL) atomicAdd(col_sum + col0 + 2 * p + h, du);
+            }
+        }
+    }
+    uint32_t word = bits << (8 * (lane & 3));
+    word |= __shfl_xor_sync(kFull, word, 1);
+    word |= __shfl_xor_sync(kFull, word, 2);
+    if ((lane & 3) == 0 && ok) mask[static_cast<size_t>(o) * (d_in >> 5) + (col0 >> 5)] = word;
+    if (ROW) {
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) sum += __shfl_xor_sync(kFull, sum, sft);
+        if (lane == 0 && o < d_out) atomicAdd(row_sum + o, sum);
+    }
+}
+
+// Programmatic dependent launch: a pack call is two kernels (pack, then the small kernel that turns sums into
+// scales).  The first lets the second be scheduled as soon as it has started and the second waits for it before it
+// touches the sums, so the second launch's latency overlaps the first kernel.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-__global__ void zero_sums_kernel(unsigned long long *__restrict__ sums, int n) {
-    grid_launch_dependents();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) sums[i] = 0ull;
-}
-
+// A CTA of 8 warps packs one tile of 32 rows x 256 columns; warp w owns rows w, w + 8, w + 16, w + 24, a lane 8
+// consecutive columns.  All eight 16-byte loads of a thread (4 rows x 2 matrices) are issued before any arithmetic,
+// a CTA makes a single round trip to memory, and four CTAs share an SM, so that one CTA's arithmetic overlaps the
+// others' loads.  (Measured and dropped: 64-row tiles with sixteen loads per thread -- half the occupancy; persistent
+// CTAs that prefetch their next tile, and one tile per warp with double-buffered batches -- several dependent round
+// trips per thread, which a 20 us kernel cannot hide; finishing a band in the CTA that draws its last ticket instead
+// of in a second kernel -- the fence and the ticket's round trip hold the whole CTA for longer than its loads take.)
+//
+// |dW| is summed in units of 2^-24, exactly.  The fp32 difference of two binary16 values is exact and a multiple of
+// 2^-24; an fp32 accumulator that starts at 0.5 and stays below 1 has an ulp of 2^-24, so adding |dW| to it is exact
+// and its bit pattern minus that of 0.5 is the sum in units.  A lane keeps one such accumulator per row (8 addends)
+// and one per column (4 addends).  An accumulator that reaches 1 (or is not finite) fails the check and that row,
+// or that warp's share of the columns, is redone by pack_row_exact in 64-bit integers; so are tiles that hang over
+// the matrix edge.
 template <bool ROW, bool COL>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_out, int d_in, int tiles_c,
             uint32_t *__restrict__ mask, unsigned long long *__restrict__ row_sum,
             unsigned long long *__restrict__ col_sum) {
     __shared__ uint32_t s_col[COL ? (kThreads / 32) * kTileCols : 1];
+    constexpr int kRowsPerWarp = kPackRows / (kThreads / 32);  // 4
+    constexpr uint32_t kHalfBits = 0x3f000000u, kOneBits = 0x3f800000u;  // bit patterns of 0.5f and 1.0f
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tile_r = blockIdx.x / tiles_c, tile_c = blockIdx.x - tile_r * tiles_c;
     const int col0 = tile_c * kTileCols + lane * 8;
-    const int row0 = tile_r * kTileRows;
-    const bool col_ok = col0 < d_in;
+    const int row0 = tile_r * kPackRows;
     const int words = d_in >> 5;
-
-    uint32_t cacc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) cacc[j] = 0;
     grid_launch_dependents();  // the finalize kernel may be scheduled; it waits for this grid
 
-#pragma unroll 4
-    for (int rr = warp; rr < kTileRows; rr += kThreads / 32) {
-        const int o = row0 + rr;
-        if (o >= d_out) break;  // warp-uniform
-        uint32_t bits = 0, fast_sum = 0;
-        unsigned long long slow_sum = 0;
-        bool slow = false;
-        uint4 a4 = make_uint4(0, 0, 0, 0), b4 = a4;
-        if (col_ok) {
-            const size_t idx = (static_cast<size_t>(o) * d_in + col0) >> 3;
-            a4 = ldg_stream(w_f + idx), b4 = ldg_stream(w_b + idx);
+    uint32_t cunits[8];  // this warp's column sums in units
+#pragma unroll
+    for (int j = 0; j < 8; ++j) cunits[j] = 0;
+    if (row0 + kPackRows <= d_out && (tile_c + 1) * kTileCols <= d_in) {  // CTA-uniform
+        uint4 a4[kRowsPerWarp], b4[kRowsPerWarp];
+#pragma unroll
+        for (int i = 0; i < kRowsPerWarp; ++i) {
+            const size_t idx = (static_cast<size_t>(row0 + warp + 8 * i) * d_in + col0) >> 3;
+            a4[i] = ldg_stream(w_f + idx);
+            b4[i] = ldg_stream(w_b + idx);
         }
-        // the first loads are in flight; nothing may be added to the sums before the kernel that zeroes them is done
-        if (rr == warp) grid_dependency_wait();
-        if (col_ok) {
-            const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
-            uint32_t spread = 0, u[8], u_or = 0;
+        float cf[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cf[j] = 0.5f;
+#pragma unroll
+        for (int i = 0; i < kRowsPerWarp; ++i) {
+            const int o = row0 + warp + 8 * i;
+            const uint32_t a[4] = {a4[i].x, a4[i].y, a4[i].z, a4[i].w}, b[4] = {b4[i].x, b4[i].y, b4[i].z, b4[i].w};
+            uint32_t spread = 0;
+            float rf = 0.5f;
 #pragma unroll
             for (int p = 0; p < 4; ++p) {
                 // bit = (w_f >= w_b): exact on binary16, false for NaN, true for -0 vs +0.  The comparison gives
                 // 0xffff per true half; pair p keeps bit 2p of the low half and bit 2p+1 of the high half.
                 const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p]));
                 spread |= ge & ((1u << (2 * p)) | (1u << (17 + 2 * p)));
-                // |dW| in units of 2^-24 by the fp32 trick.  Every binary16 is a multiple of 2^-24, so whenever
-                // |dW| < 0.5 the fp32 difference is exact and |dW| + 0.5 lies in [0.5, 1), where one ulp is 2^-24.
                 const float2 fa = __half22float2(as_half2(a[p])), fb = __half22float2(as_half2(b[p]));
-                u[2 * p] = abs_diff_units_small(fa.x, fb.x);
-                u[2 * p + 1] = abs_diff_units_small(fa.y, fb.y);
-                u_or |= u[2 * p] | u[2 * p + 1];
+                const float d0 = fabsf(__fsub_rn(fa.x, fb.x)), d1 = fabsf(__fsub_rn(fa.y, fb.y));
+                if (ROW) rf = __fadd_rn(__fadd_rn(rf, d0), d1);
+                if (COL) cf[2 * p] = __fadd_rn(cf[2 * p], d0), cf[2 * p + 1] = __fadd_rn(cf[2 * p + 1], d1);
             }
-            bits = (spread | (spread >> 16)) & 0xffu;
-            slow = (u_or & 0xff800000u) != 0;  // some |dW| >= 0.5 (or not finite): take the exact 64-bit path
-            if (!slow) {
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    if (COL) {
-                        cacc[2 * p] += u[2 * p];
-                        cacc[2 * p + 1] += u[2 * p + 1];
-                    }
-                    fast_sum += u[2 * p] + u[2 * p + 1];
+            uint32_t word = ((spread | (spread >> 16)) & 0xffu) << (8 * (lane & 3));
+            word |= __shfl_xor_sync(kFull, word, 1);
+            word |= __shfl_xor_sync(kFull, word, 2);
+            if ((lane & 3) == 0) mask[static_cast<size_t>(o) * words + (col0 >> 5)] = word;
+            if (ROW) {
+                const uint32_t rb = __float_as_uint(rf);
+                if (__all_sync(kFull, rb < kOneBits)) {  // every lane's sum stayed below 1: exact
+                    const uint32_t total = __reduce_add_sync(kFull, rb - kHalfBits);  // <= 32 * 2^23 units
+                    if (lane == 0) atomicAdd(row_sum + o, static_cast<unsigned long long>(total));
+                } else {
+                    pack_row_exact<true, false>(w_f, w_b, o, col0, d_out, d_in, mask, row_sum, col_sum, lane);
                 }
+            }
+        }
+        if (COL) {
+            uint32_t worst = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) worst = max(worst, __float_as_uint(cf[j]));
+            if (__all_sync(kFull, worst < kOneBits)) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cunits[j] = __float_as_uint(cf[j]) - kHalfBits;
             } else {
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const long long d = half_units((a[p] >> (16 * h)) & 0xffffu) -
-                                            half_units((b[p] >> (16 * h)) & 0xffffu);
-                        const unsigned long long du = static_cast<unsigned long long>(d < 0 ? -d : d);
-                        slow_sum += du;
-                        if (COL) atomicAdd(col_sum + col0 + 2 * p + h, du);
-                    }
-                }
+                for (int i = 0; i < kRowsPerWarp; ++i)
+                    pack_row_exact<false, true>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
             }
         }
-        uint32_t word = bits << (8 * (lane & 3));
-        word |= __shfl_xor_sync(kFull, word, 1);
-        word |= __shfl_xor_sync(kFull, word, 2);
-        if ((lane & 3) == 0 && col_ok) mask[static_cast<size_t>(o) * words + (col0 >> 5)] = word;
-        if (ROW) {
-            // each lane adds at most 8 * 2^23 units on the fast path, so the 32-lane sum fits 32 bits
-            unsigned long long total = __reduce_add_sync(kFull, fast_sum);
-            if (__any_sync(kFull, slow)) {
-#pragma unroll
-                for (int s = 16; s > 0; s >>= 1) slow_sum += __shfl_xor_sync(kFull, slow_sum, s);
-                total += slow_sum;
-            }
-            if (lane == 0) atomicAdd(row_sum + o, total);
-        }
+    } else {
+        for (int i = 0; i < kRowsPerWarp; ++i)
+            pack_row_exact<ROW, COL>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
     }
-    grid_dependency_wait();  // warps without a row in this tile have not waited yet
     if (COL) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s_col[warp * kTileCols + lane * 8 + j] = cacc[j];
+        for (int j = 0; j < 8; ++j) s_col[warp * kTileCols + lane * 8 + j] = cunits[j];
         __syncthreads();
         const int c = tile_c * kTileCols + threadIdx.x;
         if (c < d_in) {
-            uint32_t t = 0;  // <= 64 rows * 2^23 units
+            uint32_t sum = 0;  // <= 32 rows * 2^23 units
 #pragma unroll
-            for (int w = 0; w < kThreads / 32; ++w) t += s_col[w * kTileCols + threadIdx.x];
-            atomicAdd(col_sum + c, static_cast<unsigned long long>(t));
+            for (int w = 0; w < kThreads / 32; ++w) sum += s_col[w * kTileCols + threadIdx.x];
+            if (sum) atomicAdd(col_sum + c, static_cast<unsigned long long>(sum));
         }
     }
 }
 
-// mean = (sum * 2^-24) / n with one fp64 division, then one rounding to binary16
-__global__ void pack_finalize_kernel(const unsigned long long *__restrict__ row_sum,
-                                     const unsigned long long *__restrict__ col_sum, int d_out, int d_in,
-                                     __half *__restrict__ v_row, __half *__restrict__ v_col) {
+// Sums -> scales, and the sums go back to zero: the scratch area is left as it was found.
+__global__ void pack_finalize_kernel(unsigned long long *__restrict__ row_sum, unsigned long long *__restrict__ col_sum,
+                                     int d_out, int d_in, unsigned short *__restrict__ v_row,
+                                     unsigned short *__restrict__ v_col) {
     grid_dependency_wait();  // every tile has added its sums
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     const bool is_row = idx < d_out;
     const int j = is_row ? idx : idx - d_out;
     if (!is_row && j >= d_in) return;
-    __half *dst = is_row ? v_row : v_col;
-    if (dst == nullptr) return;
-    const unsigned long long s = is_row ? row_sum[j] : col_sum[j];
-    const double q = __ddiv_rn(static_cast<double>(s), static_cast<double>(is_row ? d_in : d_out)) *
-                     5.9604644775390625e-08;  // 2^-24, exact scaling
-    unsigned short h;
-    asm("cvt.rn.f16.f64 %0, %1;" : "=h"(h) : "d"(q));
-    reinterpret_cast<unsigned short *>(dst)[j] = h;
+    unsigned long long *src = (is_row ? row_sum : col_sum) + j;
+    unsigned short *dst = is_row ? v_row : v_col;
+    if (dst == nullptr) return;  // that axis was not asked for: its sums were never touched
+    const unsigned long long sum = *src;
+    *src = 0ull;
+    dst[j] = mean_to_half(sum, is_row ? d_in : d_out);
 }
 
 template <int AXIS>
@@ -242,39 +277,39 @@ merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *
 
 }  // namespace
 
+size_t pack_scratch_bytes(int64_t d_out, int64_t d_in) {
+    return round_up(sizeof(unsigned long long) * static_cast<size_t>(d_out + d_in), 256);
+}
+
+// scratch: pack_scratch_bytes() bytes, all zero on entry; the call leaves them zero again.
 pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
                       __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream) {
     unsigned long long *row_sum = sums, *col_sum = sums + d_out;
-    const int n = static_cast<int>(d_out + d_in);
-    zero_sums_kernel<<<(n + 255) / 256, 256, 0, stream>>>(sums, n);
     const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
-    const int64_t tiles = ((d_out + kTileRows - 1) / kTileRows) * tiles_c;
+    const int64_t tiles = ((d_out + kPackRows - 1) / kPackRows) * tiles_c;
+    if (tiles > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
+    const unsigned grid = static_cast<unsigned>(tiles);
     const uint4 *a = reinterpret_cast<const uint4 *>(w_f), *b = reinterpret_cast<const uint4 *>(w_b);
     const int n_out = static_cast<int>(d_out), n_in = static_cast<int>(d_in);
+    if (v_row && v_col)
+        pack_kernel<true, true><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    else if (v_row)
+        pack_kernel<true, false><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    else
+        pack_kernel<false, true><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+    if (cudaGetLastError() != cudaSuccess) return PD_ERR_CUDA;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled while the previous kernel runs
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled while the pack kernel runs
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(tiles));
-    cfg.blockDim = dim3(kThreads);
+    cfg.gridDim = dim3(static_cast<unsigned>((d_out + d_in + 255) / 256));
+    cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e;
-    if (v_row && v_col)
-        e = cudaLaunchKernelEx(&cfg, pack_kernel<true, true>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    else if (v_row)
-        e = cudaLaunchKernelEx(&cfg, pack_kernel<true, false>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    else
-        e = cudaLaunchKernelEx(&cfg, pack_kernel<false, true>, a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    if (e != cudaSuccess) return PD_ERR_CUDA;
-    cfg.gridDim = dim3(static_cast<unsigned>((n + 255) / 256));
-    cfg.blockDim = dim3(256);
-    if (cudaLaunchKernelEx(&cfg, pack_finalize_kernel, static_cast<const unsigned long long *>(row_sum),
-                           static_cast<const unsigned long long *>(col_sum), n_out, n_in, v_row, v_col) != cudaSuccess)
-        return PD_ERR_CUDA;
-    count_launch(3);
-    return cuda_ok(cudaGetLastError());
+    count_launch(2);
+    return cuda_ok(cudaLaunchKernelEx(&cfg, pack_finalize_kernel, row_sum, col_sum, n_out, n_in,
+                                      reinterpret_cast<unsigned short *>(v_row), reinterpret_cast<unsigned short *>(v_col)));
 }
 
 pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
@@ -335,7 +370,7 @@ extern "C" pd_status pd_pack_delta_static(const void *w_f, const void *w_b, int6
     if (!aligned16(w_f) || !aligned16(w_b) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
     unsigned long long *sums = static_sums_on_current_device();
     if (sums == nullptr) return PD_ERR_CUDA;
-    // launch_pack zero-fills sums[0 .. d_out + d_in) on the stream before the kernel adds into it
+    // the array starts zero-filled (device globals do) and every call puts what it used back to zero
     return launch_pack(static_cast<const __half *>(w_f), static_cast<const __half *>(w_b), d_out, d_in, mask,
                        static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums,
                        static_cast<cudaStream_t>(cuda_stream));

@@ -12,9 +12,8 @@ from paper_2512_19720_b200 import synth
 pytestmark = pytest.mark.gpu
 ROW, COL = 0, 1
 TOL = 5e-3
-# distinct shapes of a 70B block (q/o, k/v, gate/up, down) with the axis the paper's appendix reports as the
-# usual winner for that sub-type (k is mixed: col here so that both axes are exercised on every layer)
-SHAPES = [("q", 8192, 8192, ROW), ("k", 1024, 8192, COL), ("gate", 28672, 8192, COL), ("down", 8192, 28672, ROW)]
+# distinct shapes of a 70B block (q/o, k/v, gate/up, down); merge and both GEMVs run on both axes of every shape
+SHAPES = [("q", 8192, 8192), ("k", 1024, 8192), ("gate", 28672, 8192), ("down", 8192, 28672)]
 
 
 def dev(a):
@@ -33,8 +32,8 @@ def rel_err(y, ref):
 
 
 @pytest.mark.parametrize("layer", [0, 79])
-@pytest.mark.parametrize("name,d_out,d_in,axis", SHAPES)
-def test_build_merge_decode_70b_shapes(name, d_out, d_in, axis, layer):
+@pytest.mark.parametrize("name,d_out,d_in", SHAPES)
+def test_build_merge_decode_70b_shapes(name, d_out, d_in, layer):
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
     from paper_2512_19720_b200 import api
     w_b = synth.gen_base(d_out, d_in, 100 + layer)
@@ -50,21 +49,22 @@ def test_build_merge_decode_70b_shapes(name, d_out, d_in, axis, layer):
     assert np.array_equal(bits(g_vr), v_row.view(np.uint16))
     assert np.array_equal(bits(g_vc), v_col.view(np.uint16))
 
-    v, g_v = (v_row, g_vr) if axis == ROW else (v_col, g_vc)
-    w_hat = api.pd_merge(d_w_b, g_mask, g_v, axis)
-    torch.cuda.synchronize()
-    ref_hat = orc.merge(w_b, mask, v, axis)
-    assert np.array_equal(bits(w_hat), ref_hat.view(np.uint16))
-    del ref_hat
-
     x = synth.gen_x(1, d_in, 2000 + layer)
-    ref = orc.linear(x, w_b, mask, v, axis)
     d_x = dev(x)
-    y_fused = api.pd_linear(d_x, d_w_b, g_mask, g_v, axis)
-    y_dense = api.pd_linear(d_x, w_hat, None, None, ROW)  # the merged model: plain dense GEMV
-    torch.cuda.synchronize()
-    assert api.pd_device_status() == 0
-    assert rel_err(y_fused.cpu().numpy(), ref) <= TOL
-    assert rel_err(y_dense.cpu().numpy(), ref) <= TOL
-    del d_w_b, w_hat, g_mask
+    for axis in (ROW, COL):
+        v, g_v = (v_row, g_vr) if axis == ROW else (v_col, g_vc)
+        w_hat = api.pd_merge(d_w_b, g_mask, g_v, axis)
+        torch.cuda.synchronize()
+        ref_hat = orc.merge(w_b, mask, v, axis)
+        assert np.array_equal(bits(w_hat), ref_hat.view(np.uint16))
+        del ref_hat
+        ref = orc.linear(x, w_b, mask, v, axis)
+        y_fused = api.pd_linear(d_x, d_w_b, g_mask, g_v, axis)
+        y_dense = api.pd_linear(d_x, w_hat, None, None, ROW)  # the merged model: plain dense GEMV
+        torch.cuda.synchronize()
+        assert api.pd_device_status() == 0
+        assert rel_err(y_fused.cpu().numpy(), ref) <= TOL
+        assert rel_err(y_dense.cpu().numpy(), ref) <= TOL
+        del w_hat
+    del d_w_b, g_mask
     torch.cuda.empty_cache()

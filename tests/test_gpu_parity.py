@@ -314,11 +314,14 @@ def test_prefill_7b_m256_full(api, axis):
 
 
 @pytest.mark.parametrize("axis", [ROW, COL])
-# (4096, 4096, 512) takes 128-token tiles, (11008, 4096, 256) one 256-token tile per pair of CTAs, the others full 256-token tiles
+# every 7B shape at M = 256, 2048 and 8192 (4096 x 4096 at M = 256 is checked in full above); (4096, 4096, 512) takes
+# 128-token tiles, (11008, 4096, 256) one 256-token tile per pair of CTAs, the others full 256-token tiles.
+# Rows checked: m mod 128 in {0, 1, 127} plus 64 seeded random rows, every output column.
 @pytest.mark.parametrize("d_out,d_in,m", [(4096, 4096, 2048), (11008, 4096, 2048), (4096, 11008, 2048), (4096, 4096, 8192),
-                                          (4096, 4096, 512), (11008, 4096, 256)])
+                                          (11008, 4096, 8192), (4096, 11008, 8192), (4096, 4096, 512), (11008, 4096, 256),
+                                          (4096, 11008, 256)])
 def test_prefill_7b_sampled_rows(api, d_out, d_in, m, axis):
-    check_prefill(api, layer(d_out, d_in), m, axis, rows=synth.sample_rows(m, n_random=16))
+    check_prefill(api, layer(d_out, d_in), m, axis, rows=synth.sample_rows(m, n_random=64))
 
 
 @pytest.mark.parametrize("axis", [ROW, COL])
@@ -415,29 +418,91 @@ def test_multivariant_prefill_sized(api, d_out, d_in, n_var, m):
         assert np.max(np.abs(yh[r] - ref[r])) / np.max(np.abs(ref[r])) <= 2 * TOL
 
 
-@pytest.mark.parametrize("mixed_axes", [False, True])
-def test_multivariant_7b_shape_16_variants(api, mixed_axes):
-    # the multi-variant serving batch at full size on one 7B linear: 16 variants over one base, 64 decode rows
-    # (own id each) followed by 4 x 512 prefill rows; oracle on a fixed sample of rows
-    d_out = d_in = 4096
+def pack_variants(w_b, n_var, seed):
+    """Masks and both scale vectors of n_var fine-tunes of w_b (the oracle's pack)."""
+    d_out, d_in = w_b.shape
+    masks = np.empty((n_var, d_out, d_in // 32), dtype=np.uint32)
+    v_rows = np.empty((n_var, d_out), dtype=np.float16)
+    v_cols = np.empty((n_var, d_in), dtype=np.float16)
+    for g in range(n_var):
+        masks[g], v_rows[g], v_cols[g] = orc.pack(synth.gen_finetuned(w_b, 1000 + seed + g), w_b)
+    return masks, v_rows, v_cols
+
+
+def scales_for(axes, v_rows, v_cols):
+    n_var, d_out, d_in = len(axes), v_rows.shape[1], v_cols.shape[1]
+    vs = np.zeros((n_var, (max(d_out, d_in) + 7) // 8 * 8), dtype=np.float16)
+    for g in range(n_var):
+        if axes[g] == ROW:
+            vs[g, :d_out] = v_rows[g]
+        else:
+            vs[g, :d_in] = v_cols[g]
+    return vs
+
+
+def check_multivariant_rows(api, x, ids, w_b, masks, vs, axes, d_w_b, d_masks, rows, expect_status=0):
+    y = api.pd_linear_multivariant(dev(x), dev(ids), d_w_b, d_masks, dev(vs), axes)
+    y2 = api.pd_linear_multivariant(dev(x), dev(ids), d_w_b, d_masks, dev(vs), axes)
+    torch.cuda.synchronize()
+    assert api.pd_device_status() == expect_status
+    assert torch.equal(y[rows], y2[rows]), "two runs must be bit-identical"
+    ref, _ = orc.linear_multivariant(np.ascontiguousarray(x[rows]), np.ascontiguousarray(ids[rows]), w_b, masks, vs, axes)
+    yh = host(y).astype(np.float64)
+    assert np.isfinite(yh[rows]).all()
+    assert rel_err(yh[rows], ref) <= TOL
+    for i, r in enumerate(rows):  # row by row: no row may borrow another variant's delta
+        assert np.max(np.abs(yh[r] - ref[i])) / np.max(np.abs(ref[i])) <= 2 * TOL
+
+
+# the multi-variant serving batch at full size on every 7B shape: 16 variants over one base; 64 decode rows (own id
+# each), 64 + 4 x 512 rows with an id per row, and the same with one id per 512-row sequence; uniform row axis
+# (both per-row batches), uniform col axis (decode batch) and mixed axes (decode batch and per-sequence batch);
+# oracle on all 64 decode rows / on m mod 128 in {0, 1, 127} plus 64 random rows
+@pytest.mark.parametrize("d_out,d_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_multivariant_7b_shapes_16_variants(api, d_out, d_in):
     n_var = 16
     w_b = synth.gen_base(d_out, d_in, 31)
-    masks, vs, axes = make_variants(w_b, n_var, 31, mixed_axes=mixed_axes, axis=ROW)
-    d_args = (dev(w_b), dev(masks), dev(vs))
-    for m, ids in ((64, synth.gen_ids(64, n_var, 33)), (2112, synth.gen_ids(2112, n_var, 34)),
-                   (2112, synth.gen_ids_per_sequence(64, 4, 512, n_var, 35))):
-        x = synth.gen_x(m, d_in, 32 + m)
-        y = api.pd_linear_multivariant(dev(x), dev(ids), d_args[0], d_args[1], d_args[2], axes)
-        torch.cuda.synchronize()
-        assert api.pd_device_status() == 0
-        rows = np.arange(m) if m <= 64 else synth.sample_rows(m, n_random=24)
-        ref, bad = orc.linear_multivariant(np.ascontiguousarray(x[rows]), np.ascontiguousarray(ids[rows]), w_b, masks, vs, axes)
-        assert bad == 0
-        yh = host(y).astype(np.float64)
-        assert np.isfinite(yh).all()
-        assert rel_err(yh[rows], ref) <= TOL
-        for i, r in enumerate(rows):  # row by row: no row may borrow another variant's delta
-            assert np.max(np.abs(yh[r] - ref[i])) / np.max(np.abs(ref[i])) <= 2 * TOL
+    masks, v_rows, v_cols = pack_variants(w_b, n_var, 31)
+    d_w_b, d_masks = dev(w_b), dev(masks)
+    batches = [(64, synth.gen_ids(64, n_var, 33)), (2112, synth.gen_ids(2112, n_var, 34)),
+               (2112, synth.gen_ids_per_sequence(64, 4, 512, n_var, 35))]
+    plan = (("row", [ROW] * n_var, batches[:2]), ("col", [COL] * n_var, batches[:1]),
+            ("mixed", [g % 2 for g in range(n_var)], batches[::2]))
+    for name, axes, todo in plan:
+        axes = np.array(axes, dtype=np.uint8)
+        vs = scales_for(axes, v_rows, v_cols)
+        for m, ids in todo:
+            x = synth.gen_x(m, d_in, 32 + m)
+            rows = np.arange(m) if m <= 64 else synth.sample_rows(m, n_random=64)
+            check_multivariant_rows(api, x, ids, w_b, masks, vs, axes, d_w_b, d_masks, rows)
+    del d_w_b, d_masks
+    torch.cuda.empty_cache()
+
+
+# decode-sized batches through the one-pass kernel: few rows, few or many variants, ids of -1, mixed axes,
+# more than eight rows of one variant, more items than one pass holds
+@pytest.mark.parametrize("d_out,d_in", [(1024, 1024), (4096, 4096)])
+def test_multivariant_decode_batches(api, d_out, d_in):
+    w_b = synth.gen_base(d_out, d_in, 41)
+    masks, v_rows, v_cols = pack_variants(w_b, 16, 41)
+    d_w_b = dev(w_b)
+    for m, n_var, seed in ((5, 4, 1), (16, 4, 2), (16, 16, 3), (5, 16, 4), (1, 16, 5), (40, 2, 6), (64, 16, 7)):
+        axes = np.array([g % 2 for g in range(n_var)], dtype=np.uint8)
+        vs = scales_for(axes, v_rows[:n_var], v_cols[:n_var])
+        ids = synth.gen_ids(m, n_var, 50 + seed)
+        if m >= 5:
+            ids[1] = -1
+            ids[m - 1] = -1
+        x = synth.gen_x(m, d_in, 60 + seed)
+        check_multivariant_rows(api, x, ids, w_b, masks[:n_var], vs, axes, d_w_b, dev(masks[:n_var]), np.arange(m))
+    # 64 rows over 64 variants: 64 items, four passes
+    if d_out == 1024:
+        masks64 = np.concatenate([masks] * 4)
+        axes = np.array([g % 2 for g in range(64)], dtype=np.uint8)
+        vs = scales_for(axes, np.concatenate([v_rows] * 4), np.concatenate([v_cols] * 4))
+        ids = np.arange(64, dtype=np.int32)[::-1].copy()
+        x = synth.gen_x(64, d_in, 70)
+        check_multivariant_rows(api, x, ids, w_b, masks64, vs, axes, d_w_b, dev(masks64), np.arange(64))
 
 
 def test_multivariant_bad_id_is_latched(api):
@@ -452,6 +517,76 @@ def test_multivariant_bad_id_is_latched(api):
     assert bad == 1
     keep = [0, 1, 3, 4, 5]
     assert rel_err(host(y)[keep], ref[keep]) <= TOL
+
+
+@pytest.mark.parametrize("m", [40, 100])
+def test_multivariant_bad_id_in_a_larger_batch(api, m):
+    # one id out of range among m rows, on a private zero-filled workspace: m = 40 runs the one-pass decode kernel,
+    # m = 100 the sorted tensor-core path (whose gather must skip the row that belongs to no bucket).  The call
+    # latches PD_ERR_BAD_VARIANT and every other row is still right.
+    d_out, d_in, n_var = 256, 512, 3
+    w_b = synth.gen_base(d_out, d_in, 16)
+    masks, vs, axes = make_variants(w_b, n_var, 16)
+    x = synth.gen_x(m, d_in, 17)
+    ids = synth.gen_ids(m, n_var, 18)
+    ids[7] = n_var + 4
+    ws = torch.zeros(api.workspace_bytes(api.OP_LINEAR_MULTIVARIANT, m, n_var, d_out, d_in), dtype=torch.uint8, device="cuda")
+    y = api.pd_linear_multivariant(dev(x), dev(ids), dev(w_b), dev(masks), dev(vs), axes, workspace=ws)
+    assert api.pd_device_status(workspace=ws) == 6  # PD_ERR_BAD_VARIANT
+    assert api.pd_device_status(workspace=ws) == 0
+    ref, bad = orc.linear_multivariant(x, ids, w_b, masks, vs, axes)
+    assert bad == 1
+    keep = [r for r in range(m) if r != 7]
+    assert rel_err(host(y)[keep], ref[keep]) <= TOL
+
+
+# ------------------------------------------------------------------ stream order, failure path
+def test_linear_right_after_pack_and_merge_on_one_stream(api):
+    # pd_pack_delta -> pd_linear and pd_merge -> pd_linear(w_hat, mask = NULL), queued back to back with no
+    # synchronisation in between and with the intermediate buffers full of garbage beforehand: the decode kernel
+    # may start early (programmatic dependent launch) but must not read the weights before they are written
+    for d_out, d_in in ((4096, 4096), (1024, 1024)):
+        L = layer(d_out, d_in)
+        x = synth.gen_x(4, d_in, 80)
+        d_x = dev(x)
+        for axis in (ROW, COL):
+            ref = orc.linear(x, L.w_b, L.mask, L.v(axis), axis)
+            merged = orc.merge(L.w_b, L.mask, L.v(axis), axis)
+            ref_dense = x.astype(np.float64) @ merged.astype(np.float64).T
+            for rep in range(3):
+                mask = torch.full((d_out, d_in // 32), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+                v_row = torch.full((d_out,), 77.0, dtype=torch.float16, device="cuda")
+                v_col = torch.full((d_in,), 77.0, dtype=torch.float16, device="cuda")
+                w_hat = torch.full((d_out, d_in), 55.0, dtype=torch.float16, device="cuda")
+                torch.cuda.synchronize()
+                api.pd_pack_delta(L.d_w_f, L.d_w_b, mask=mask, v_row=v_row, v_col=v_col)
+                y = api.pd_linear(d_x, L.d_w_b, mask, v_row if axis == ROW else v_col, axis)
+                api.pd_merge(L.d_w_b, mask, v_row if axis == ROW else v_col, axis, w_hat=w_hat)
+                y_dense = api.pd_linear(d_x, w_hat, None, None, ROW)
+                torch.cuda.synchronize()
+                assert api.pd_device_status() == 0
+                assert rel_err(host(y), ref) <= TOL
+                assert rel_err(host(y_dense), ref_dense) <= TOL
+    # the resident-weights flag gives the same numbers when the weights really are resident
+    L = layer(1024, 1024)
+    x = synth.gen_x(16, 1024, 81)
+    y0 = api.pd_linear(dev(x), L.d_w_b, L.d_mask, L.d_v_row, ROW)
+    y1 = api.pd_linear(dev(x), L.d_w_b, L.d_mask, L.d_v_row, ROW, weights_resident=True)
+    torch.cuda.synchronize()
+    assert torch.equal(y0, y1)
+
+
+def test_bounded_wait_runs_out_and_is_reported(api):
+    # a wait that nothing satisfies gives up after its limit, latches PD_ERR_DEVICE_TIMEOUT and the kernel returns;
+    # the context stays usable
+    ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    api.pd_selftest_bounded_wait(100000, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(ws[4:8].view(torch.int32).item()) == 99  # the detail word names the wait that gave up
+    assert api.pd_device_status(workspace=ws) == 7  # PD_ERR_DEVICE_TIMEOUT
+    assert api.pd_device_status(workspace=ws) == 0  # reading it clears it
+    L = layer(1024, 1024)
+    check_linear(api, L, 4, ROW)
 
 
 def test_native_library_is_the_one_in_tree(api):

@@ -4,7 +4,7 @@ It serves callers that cannot get scratch memory when they pack a layer (a fixed
 a plug-in that must not touch the CUDA allocator, code running while a stream is captured).
 Its scratch is one array inside the library that every call on the GPU shares, so the test makes
 two calls in a row on different layers -- the second would inherit the first one's sums if the
-array were not cleared -- and requires both to equal pd_pack_delta bit for bit.
+array were not cleared -- and requires both to equal pd_pack_delta, and the CPU oracle, bit for bit.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import pd_oracle as orc
 from paper_2512_19720_b200 import synth
 
 
@@ -25,11 +26,12 @@ def test_static_pack_matches_workspace_pack_on_two_calls_in_a_row():
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
     from paper_2512_19720_b200 import api
 
-    layers = []
+    layers, expected = [], []
     for (d_out, d_in), seed in (((1024, 1024), 21), ((200, 1056), 22)):
         w_b = synth.gen_base(d_out, d_in, seed)
         w_f = synth.gen_finetuned(w_b, 1000 + seed)
         layers.append((_dev(w_f), _dev(w_b)))
+        expected.append(orc.pack(w_f, w_b))
 
     # outputs are allocated up front: the calls under test receive only existing tensors
     outs = []
@@ -44,12 +46,15 @@ def test_static_pack_matches_workspace_pack_on_two_calls_in_a_row():
         api.pd_pack_delta_static(w_f, w_b, mask, v_row, v_col)
     torch.cuda.synchronize()
 
-    for (w_f, w_b), (mask, v_row, v_col) in zip(layers, outs):
+    for (w_f, w_b), (mask, v_row, v_col), (o_mask, o_row, o_col) in zip(layers, outs, expected):
         ref_mask, ref_row, ref_col = api.pd_pack_delta(w_f, w_b)
         torch.cuda.synchronize()
         assert torch.equal(mask, ref_mask)
         assert torch.equal(v_row.view(torch.int16), ref_row.view(torch.int16))
         assert torch.equal(v_col.view(torch.int16), ref_col.view(torch.int16))
+        assert np.array_equal(mask.cpu().numpy().view(np.uint32), o_mask)  # and the CPU oracle
+        assert np.array_equal(v_row.cpu().numpy().view(np.uint16), o_row.view(np.uint16))
+        assert np.array_equal(v_col.cpu().numpy().view(np.uint16), o_col.view(np.uint16))
 
     # one axis only, and again over the array the calls above left dirty
     w_f, w_b = layers[0]
@@ -61,6 +66,8 @@ def test_static_pack_matches_workspace_pack_on_two_calls_in_a_row():
 
 
 def test_static_pack_rejects_sizes_beyond_its_array():
+    from paper_2512_19720_b200 import build
+    build.build()
     from paper_2512_19720_b200 import api
     a = 0x10000  # never dereferenced: the size check comes before any launch
     before = api.launch_count()
