@@ -68,6 +68,45 @@ def gen_finetuned(w_b: np.ndarray, seed: int, sigma: float = 1e-3) -> np.ndarray
     return w_f
 
 
+def to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """float32 array -> bfloat16 bit patterns (uint16), round to nearest even (storage conversion only)."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    return u.astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns -> the float32 values they denote (exact)."""
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def gen_base_bf16(d_out: int, d_in: int, seed: int = 0) -> np.ndarray:
+    """Base weights as bfloat16 bit patterns [d_out, d_in], entries ~ N(0, 0.02^2) (the draws of gen_base)."""
+    z = _rng(seed, TAG_BASE).standard_normal((d_out, d_in), dtype=np.float32)
+    z *= np.float32(0.02)
+    return to_bf16_bits(z)
+
+
+def gen_finetuned_bf16(w_b: np.ndarray, seed: int, sigma: float = 1e-3) -> np.ndarray:
+    """Fine-tuned weights W_f = bf16(W_b + sigma * s_r[o] * z) as bfloat16 bit patterns."""
+    d_out, d_in = w_b.shape
+    s_r = gen_row_spread(d_out, seed).astype(np.float32)
+    rng = _rng(seed, TAG_DELTA)
+    w_f = np.empty_like(w_b)
+    rows = max(1, (1 << 24) // d_in)
+    for r0 in range(0, d_out, rows):
+        r1 = min(d_out, r0 + rows)
+        z = rng.standard_normal((r1 - r0, d_in), dtype=np.float32)
+        z *= (np.float32(sigma) * s_r[r0:r1])[:, None]
+        w_f[r0:r1] = to_bf16_bits((bf16_bits_to_f32(w_b[r0:r1]).astype(np.float64) + z.astype(np.float64)).astype(np.float32))
+    return w_f
+
+
+def gen_x_bf16(m: int, d_in: int, seed: int = 2000) -> np.ndarray:
+    """Activations as bfloat16 bit patterns [M, d_in], entries ~ N(0,1)."""
+    return to_bf16_bits(_rng(seed, TAG_X).standard_normal((m, d_in), dtype=np.float32))
+
+
 def gen_x(m: int, d_in: int, seed: int = 2000) -> np.ndarray:
     """Activations x, fp16 [M, d_in], entries ~ N(0,1)."""
     return _rng(seed, TAG_X).standard_normal((m, d_in), dtype=np.float32).astype(np.float16)
