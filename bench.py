@@ -10,6 +10,7 @@ A step is one pass of the whole path, all through the C ABI, inputs resident in 
     multi_*        pd_linear_multivariant, 16 variants over one base: 64 decode rows; 64 + 4 x 512 rows with an id
                    per row; the same with one id per 512-row sequence; both batch sizes with mixed axes
     merge          pd_merge on the 7 linears, row and col
+    bf16_*         pack, decode (M in {1, 4, 16}), prefill (M = 2048) and merge with bfloat16 weights and activations
   single 1024 x 1024 layer
     c1_*           pd_linear at M = 1 and 16 over 128 rotated copies (weights from HBM) and on one copy (L2-resident)
   Llama-70B-shaped block, 80 layers streamed through one set of per-layer buffers
@@ -312,6 +313,16 @@ def run_ours(args):
                             v_col=torch.empty(d_in, dtype=torch.float16, device=dev)))
         big_x = synth_torch.gen_x(1, 28672, 2070, dev)
         big_y = torch.empty((1, 28672), dtype=torch.float16, device=dev)
+    # BF16 variants: the same block with base, fine-tune and activations in bfloat16
+    bf_layers = []
+    for li, (name, d_out, d_in) in enumerate(BLOCK):
+        w_b = synth_torch.gen_base(d_out, d_in, 10 + li, dev).bfloat16()
+        w_f = synth_torch.gen_finetuned(w_b, 100 + li)
+        mask, v_row, v_col = api.pd_pack_delta(w_f, w_b)
+        bf_layers.append(dict(name=name, d_out=d_out, d_in=d_in, w_b=w_b, w_f=w_f, mask=mask, v=(v_row, v_col),
+                              w_hat=torch.empty_like(w_b)))
+    bf_x = {d_in: x_all[d_in][:2048].bfloat16() for d_in in x_all}
+    bf_y = {d_out: torch.empty((2048, d_out), dtype=torch.bfloat16, device=dev) for d_out in y_all}
     torch.cuda.synchronize()
 
     # ---- sections: name -> (body, algorithmic work, unit, calls, kernel label)
@@ -332,6 +343,22 @@ def run_ours(args):
     def run_merge():
         for axis in (ROW, COL):
             for L in layers:
+                api.pd_merge(L["w_b"], L["mask"], L["v"][axis], axis, w_hat=L["w_hat"])
+
+    def bf_pack():
+        for L in bf_layers:
+            api.pd_pack_delta(L["w_f"], L["w_b"], mask=L["mask"], v_row=L["v"][0], v_col=L["v"][1])
+
+    def bf_linear(ms, resident):
+        for m in ms:
+            for axis in (ROW, COL):
+                for L in bf_layers:
+                    api.pd_linear(bf_x[L["d_in"]][:m], L["w_b"], L["mask"], L["v"][axis], axis, y=bf_y[L["d_out"]][:m],
+                                  weights_resident=resident)
+
+    def bf_merge():
+        for axis in (ROW, COL):
+            for L in bf_layers:
                 api.pd_merge(L["w_b"], L["mask"], L["v"][axis], axis, w_hat=L["w_hat"])
 
     def run_c1(m, rotated):
@@ -382,6 +409,11 @@ def run_ours(args):
         "TFLOP/s", 7, "gemm_pair_kernel<grouped>")
     add("merge", run_merge, sum(merge_bytes(L["d_out"], L["d_in"], ax) for ax in (ROW, COL) for L in layers), "GB/s", 14,
         "merge_kernel")
+    add("bf16_pack", bf_pack, S["pack"]["work"], "GB/s", 7, "pack_kernel<bf16>")
+    add("bf16_decode", lambda: bf_linear(DECODE_M, True), sum(S[f"decode_m{m}"]["work"] for m in DECODE_M), "GB/s", 42,
+        "gemv_stream_kernel<bf16>")
+    add("bf16_prefill_m2048", lambda: bf_linear((2048,), False), 2 * flops(2048), "TFLOP/s", 14, "gemm_pair_kernel<bf16>")
+    add("bf16_merge", bf_merge, S["merge"]["work"], "GB/s", 14, "merge_kernel<bf16>")
     for m in (1, 16):
         for rotated in (True, False):
             add(f"c1_m{m}_{'rotated' if rotated else 'resident'}", lambda m=m, r=rotated: run_c1(m, r),

@@ -176,6 +176,39 @@ pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis
                    int64_t d_out, int64_t d_in, void *w_hat, void *cuda_stream);
 
 /*
+ * BF16 variants -- the same four operations with the base, the fine-tuned weights, the activations and the outputs
+ * in bfloat16 (the upper 16 bits of an IEEE binary32, passed as void*); masks, ids and the binary16 scale vectors
+ * are unchanged.
+ * Paper: Implementation remarks -- the base weights are "kept as (in,out) BF16", the calibration inputs and outputs
+ * are stored as BF16 tensors and the scale vectors in FP16.
+ *
+ *   pd_pack_delta_bf16 : bit = (w_f >= w_b), an exact comparison.  The scales are means of floor(|dW| * 2^24)
+ *       units of 2^-24 -- bfloat16 differences are not multiples of one small unit, so |dW| is cut down to that grid
+ *       before it is summed; the sum is an integer and does not depend on order (for binary16 inputs the grid holds
+ *       |dW| exactly, which is what pd_pack_delta sums).  One fp64 division, one rounding to binary16.  Exact while
+ *       |w| <= 2^28 and a sum of |dW| stays below 2^29.
+ *   pd_merge_bf16      : w_hat = bf16( fp32(w_b) + (+-)fp32(v) ): one binary32 addition, one rounding to bfloat16.
+ *   pd_linear_bf16     : as pd_linear_ex.  W_hat = W_b +- v is formed on chip in bfloat16: v is rounded to bfloat16
+ *       once, then one bfloat16 addition; bfloat16 products accumulate in fp32 and y is rounded to bfloat16 once.
+ *   pd_linear_multivariant_bf16 : as pd_linear_multivariant.
+ * Arguments, alignment rules, workspaces and error behaviour are those of the binary16 calls.
+ */
+pd_status pd_pack_delta_bf16(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in,
+                             uint32_t *mask, void *v_row, void *v_col,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+pd_status pd_merge_bf16(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
+                        int64_t d_out, int64_t d_in, void *w_hat, void *cuda_stream);
+pd_status pd_linear_bf16(const void *x, int64_t M, int64_t ldx,
+                         const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
+                         int64_t d_out, int64_t d_in, void *y, int64_t ldy,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream, uint32_t flags);
+pd_status pd_linear_multivariant_bf16(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids,
+                                      const void *w_b, const uint32_t *masks, const void *vs,
+                                      int64_t v_stride, const uint8_t *axes, int32_t V,
+                                      int64_t d_out, int64_t d_in, void *y, int64_t ldy,
+                                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * pd_pack_delta_static -- pd_pack_delta without a workspace argument and without any allocation.
  * The paper has no counterpart: this entry point exists for the library's users, not the method.
  *

@@ -19,7 +19,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpd.so")
 
 EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_ex", "pd_linear_multivariant", "pd_merge",
-           "pd_workspace_bytes", "pd_device_status", "pd_status_string", "pd_launch_count", "pd_selftest_bounded_wait"]
+           "pd_workspace_bytes", "pd_device_status", "pd_status_string", "pd_launch_count", "pd_selftest_bounded_wait",
+           "pd_pack_delta_bf16", "pd_merge_bf16", "pd_linear_bf16", "pd_linear_multivariant_bf16"]
 LINEAR_WEIGHTS_RESIDENT = 1
 
 
@@ -59,6 +60,11 @@ def _load() -> ctypes.CDLL:
     lib.pd_status_string.restype = ctypes.c_char_p
     lib.pd_launch_count.argtypes = []
     lib.pd_launch_count.restype = i64
+    for name, proto in (("pd_pack_delta_bf16", lib.pd_pack_delta), ("pd_merge_bf16", lib.pd_merge),
+                        ("pd_linear_bf16", lib.pd_linear_ex), ("pd_linear_multivariant_bf16", lib.pd_linear_multivariant)):
+        fn = getattr(lib, name)
+        fn.argtypes, fn.restype = proto.argtypes, ctypes.c_int
+        assert fn.argtypes is not None
     return lib
 
 
@@ -122,10 +128,18 @@ def _want(t, dtype, name):
         raise TypeError(f"{name} must be a CUDA tensor of {dtype}")
 
 
+def _elem(t, name):
+    """True for bfloat16 weights / activations, False for float16 (the two storage types the library has)."""
+    if not t.is_cuda or t.dtype not in (torch.float16, torch.bfloat16):
+        raise TypeError(f"{name} must be a CUDA tensor of float16 or bfloat16")
+    return t.dtype == torch.bfloat16
+
+
 def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None, v_col=None, workspace=None):
     """mask uint32-as-int32 [d_out, d_in/32], v_row fp16 [d_out] | None, v_col fp16 [d_in] | None.
     A workspace passed in must be all zero (the call leaves it so)."""
-    _want(w_f, torch.float16, "w_f"), _want(w_b, torch.float16, "w_b")
+    bf16 = _elem(w_b, "w_b")
+    _want(w_f, w_b.dtype, "w_f")
     assert w_f.shape == w_b.shape and w_f.is_contiguous() and w_b.is_contiguous()
     d_out, d_in = w_b.shape
     dev = w_b.device
@@ -137,9 +151,9 @@ def pd_pack_delta(w_f, w_b, want_row=True, want_col=True, mask=None, v_row=None,
         v_col = torch.empty(d_in, dtype=torch.float16, device=dev)
     need = workspace_bytes(OP_PACK, 0, 0, d_out, d_in)
     ws = workspace if workspace is not None else _pack_workspace(need, dev)
-    _check(lib.pd_pack_delta(_ptr(w_f), _ptr(w_b), d_out, d_in, _ptr(mask), _ptr(v_row if want_row else None),
-                             _ptr(v_col if want_col else None), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
-           "pd_pack_delta")
+    fn = lib.pd_pack_delta_bf16 if bf16 else lib.pd_pack_delta
+    _check(fn(_ptr(w_f), _ptr(w_b), d_out, d_in, _ptr(mask), _ptr(v_row if want_row else None),
+              _ptr(v_col if want_col else None), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pd_pack_delta")
     return mask, (v_row if want_row else None), (v_col if want_col else None)
 
 
@@ -159,18 +173,21 @@ def pd_pack_delta_static(w_f, w_b, mask, v_row=None, v_col=None):
 def pd_linear(x, w_b, mask, v, axis, y=None, workspace=None, weights_resident=False):
     """y fp16 [M, d_out] = x . (W_b + v (.) B)^T; mask None = base weights only.  weights_resident=True passes
     PD_LINEAR_WEIGHTS_RESIDENT: no earlier work on the stream writes w_b, mask or v."""
-    _want(x, torch.float16, "x"), _want(w_b, torch.float16, "w_b")
+    bf16 = _elem(w_b, "w_b")
+    _want(x, w_b.dtype, "x")
     assert x.dim() == 2 and x.stride(1) == 1 and w_b.is_contiguous()
     m, d_in = x.shape
     d_out = w_b.shape[0]
     assert w_b.shape[1] == d_in
     if y is None:
-        y = torch.empty((m, d_out), dtype=torch.float16, device=x.device)
+        y = torch.empty((m, d_out), dtype=w_b.dtype, device=x.device)
+    assert y.dtype == w_b.dtype
     need = workspace_bytes(OP_LINEAR, m, 0, d_out, d_in)
     ws = workspace if workspace is not None else _workspace(need, x.device)
-    _check(lib.pd_linear_ex(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
-                            y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
-                            LINEAR_WEIGHTS_RESIDENT if weights_resident else 0), "pd_linear")
+    fn = lib.pd_linear_bf16 if bf16 else lib.pd_linear_ex
+    _check(fn(_ptr(x), m, x.stride(0), _ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(y),
+              y.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream(),
+              LINEAR_WEIGHTS_RESIDENT if weights_resident else 0), "pd_linear")
     return y
 
 
@@ -193,30 +210,34 @@ def pd_linear_host(x_host, x_dev, w_b, mask, v, axis, y_dev, y_host, workspace=N
 def pd_linear_multivariant(x, variant_ids, w_b, masks, vs, axes, y=None, workspace=None):
     """Row m of x uses variant variant_ids[m] (-1 = base only).  masks [V, d_out, d_in/32], vs fp16
     [V, v_stride], axes: sequence of V axis codes (host)."""
-    _want(x, torch.float16, "x"), _want(w_b, torch.float16, "w_b"), _want(variant_ids, torch.int32, "variant_ids")
+    bf16 = _elem(w_b, "w_b")
+    _want(x, w_b.dtype, "x"), _want(variant_ids, torch.int32, "variant_ids"), _want(vs, torch.float16, "vs")
     assert x.dim() == 2 and x.stride(1) == 1 and w_b.is_contiguous() and masks.is_contiguous() and vs.is_contiguous()
     m, d_in = x.shape
     d_out = w_b.shape[0]
     n_var = masks.shape[0]
     if y is None:
-        y = torch.empty((m, d_out), dtype=torch.float16, device=x.device)
+        y = torch.empty((m, d_out), dtype=w_b.dtype, device=x.device)
+    assert y.dtype == w_b.dtype
     axes_arr = (ctypes.c_uint8 * n_var)(*[int(a) for a in axes])
     need = workspace_bytes(OP_LINEAR_MULTIVARIANT, m, n_var, d_out, d_in)
     ws = workspace if workspace is not None else _workspace(need, x.device)
-    _check(lib.pd_linear_multivariant(_ptr(x), m, x.stride(0), _ptr(variant_ids), _ptr(w_b), _ptr(masks), _ptr(vs),
-                                      vs.stride(0), axes_arr, n_var, d_out, d_in, _ptr(y), y.stride(0), _ptr(ws),
-                                      ws.numel() * ws.element_size(), _stream()), "pd_linear_multivariant")
+    fn = lib.pd_linear_multivariant_bf16 if bf16 else lib.pd_linear_multivariant
+    _check(fn(_ptr(x), m, x.stride(0), _ptr(variant_ids), _ptr(w_b), _ptr(masks), _ptr(vs),
+              vs.stride(0), axes_arr, n_var, d_out, d_in, _ptr(y), y.stride(0), _ptr(ws),
+              ws.numel() * ws.element_size(), _stream()), "pd_linear_multivariant")
     return y
 
 
 def pd_merge(w_b, mask, v, axis, w_hat=None):
     """Dense fp16 W_hat = fp16(fp32(W_b) +- fp32(v)); w_hat may be w_b itself."""
-    _want(w_b, torch.float16, "w_b")
+    bf16 = _elem(w_b, "w_b")
     assert w_b.is_contiguous()
     d_out, d_in = w_b.shape
     if w_hat is None:
         w_hat = torch.empty_like(w_b)
-    _check(lib.pd_merge(_ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(w_hat), _stream()), "pd_merge")
+    assert w_hat.dtype == w_b.dtype
+    _check((lib.pd_merge_bf16 if bf16 else lib.pd_merge)(_ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(w_hat), _stream()), "pd_merge")
     return w_hat
 
 

@@ -190,8 +190,12 @@ const char *pd_status_string(pd_status s) {
 
 int64_t pd_launch_count(void) { return g_launches.load(); }
 
-pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in, uint32_t *mask, void *v_row,
-                        void *v_col, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+pd_status pack_impl(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in, uint32_t *mask, void *v_row,
+                    void *v_col, void *workspace, size_t workspace_bytes, void *cuda_stream, bool bf16) {
     if (!w_f || !w_b || !mask || (!v_row && !v_col) || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
     if (d_in % 32 != 0 || d_out > INT_MAX / 2 || d_in > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(w_f) || !aligned16(w_b) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
@@ -199,30 +203,24 @@ pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t
         return PD_ERR_WORKSPACE;
     auto *sums = reinterpret_cast<unsigned long long *>(static_cast<unsigned char *>(workspace) + kStatusBytes);
     return launch_pack(static_cast<const __half *>(w_f), static_cast<const __half *>(w_b), d_out, d_in, mask,
-                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums,
+                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums, bf16,
                        static_cast<cudaStream_t>(cuda_stream));
 }
 
-pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis, int64_t d_out, int64_t d_in,
-                   void *w_hat, void *cuda_stream) {
+pd_status merge_impl(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis, int64_t d_out, int64_t d_in,
+                     void *w_hat, void *cuda_stream, bool bf16) {
     if (!w_b || !mask || !v || !w_hat || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
     if (axis != PD_AXIS_ROW && axis != PD_AXIS_COL) return PD_ERR_INVALID_ARG;
     if (d_in % 32 != 0 || d_out > INT_MAX / 2 || d_in > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(w_b) || !aligned16(w_hat) || (reinterpret_cast<uintptr_t>(mask) & 3u)) return PD_ERR_ALIGNMENT;
     if (axis == PD_AXIS_COL && !aligned16(v)) return PD_ERR_ALIGNMENT;
     return launch_merge(static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis, d_out, d_in,
-                        static_cast<__half *>(w_hat), static_cast<cudaStream_t>(cuda_stream));
+                        static_cast<__half *>(w_hat), bf16, static_cast<cudaStream_t>(cuda_stream));
 }
 
-pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
-                    pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
-                    size_t workspace_bytes, void *cuda_stream) {
-    return pd_linear_ex(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, workspace, workspace_bytes, cuda_stream, 0u);
-}
-
-pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
-                       pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
-                       size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
+pd_status linear_impl(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                      pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                      size_t workspace_bytes, void *cuda_stream, uint32_t flags, bool bf16) {
     pd_status st = check_matrix_args(x, M, ldx, w_b, d_out, d_in, y, ldy);
     if (st != PD_OK) return st;
     if (flags & ~static_cast<uint32_t>(PD_LINEAR_WEIGHTS_RESIDENT)) return PD_ERR_INVALID_ARG;
@@ -236,10 +234,11 @@ pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx, const void *w_b, c
     __half *yh = static_cast<__half *>(y);
     if (M > kGemvMaxTokens && d_in >= 64)  // narrower layers would need a TMA box wider than the matrix
         return launch_gemm(xh, M, ldx, static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis,
-                           d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), stream);
+                           d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), bf16, stream);
     GemvScratch scratch;
     scratch.status = static_cast<uint32_t *>(workspace);
     scratch.weights_resident = (flags & PD_LINEAR_WEIGHTS_RESIDENT) != 0;
+    scratch.bf16 = bf16;
     for (int64_t m0 = 0; m0 < M; m0 += 16) {
         const int rows = static_cast<int>(M - m0 < 16 ? M - m0 : 16);
         st = launch_gemv(xh + m0 * ldx, rows, ldx, static_cast<const __half *>(w_b), mask,
@@ -250,6 +249,61 @@ pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx, const void *w_b, c
     return PD_OK;
 }
 
+pd_status multivariant_impl(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
+                            const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes, int32_t V,
+                            int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream, bool bf16);
+
+}  // namespace
+
+extern "C" {
+
+pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in, uint32_t *mask, void *v_row,
+                        void *v_col, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return pack_impl(w_f, w_b, d_out, d_in, mask, v_row, v_col, workspace, workspace_bytes, cuda_stream, false);
+}
+pd_status pd_pack_delta_bf16(const void *w_f, const void *w_b, int64_t d_out, int64_t d_in, uint32_t *mask, void *v_row,
+                             void *v_col, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return pack_impl(w_f, w_b, d_out, d_in, mask, v_row, v_col, workspace, workspace_bytes, cuda_stream, true);
+}
+pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis, int64_t d_out, int64_t d_in,
+                   void *w_hat, void *cuda_stream) {
+    return merge_impl(w_b, mask, v, axis, d_out, d_in, w_hat, cuda_stream, false);
+}
+pd_status pd_merge_bf16(const void *w_b, const uint32_t *mask, const void *v, pd_axis axis, int64_t d_out, int64_t d_in,
+                        void *w_hat, void *cuda_stream) {
+    return merge_impl(w_b, mask, v, axis, d_out, d_in, w_hat, cuda_stream, true);
+}
+pd_status pd_linear(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                    pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                    size_t workspace_bytes, void *cuda_stream) {
+    return linear_impl(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, workspace, workspace_bytes, cuda_stream, 0u, false);
+}
+pd_status pd_linear_ex(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                       pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
+    return linear_impl(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, workspace, workspace_bytes, cuda_stream, flags, false);
+}
+pd_status pd_linear_bf16(const void *x, int64_t M, int64_t ldx, const void *w_b, const uint32_t *mask, const void *v,
+                         pd_axis axis, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                         size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
+    return linear_impl(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, workspace, workspace_bytes, cuda_stream, flags, true);
+}
+pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
+                                 const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes,
+                                 int32_t V, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                                 size_t workspace_bytes, void *cuda_stream) {
+    return multivariant_impl(x, M, ldx, variant_ids, w_b, masks, vs, v_stride, axes, V, d_out, d_in, y, ldy, workspace,
+                             workspace_bytes, cuda_stream, false);
+}
+pd_status pd_linear_multivariant_bf16(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
+                                      const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes,
+                                      int32_t V, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
+                                      size_t workspace_bytes, void *cuda_stream) {
+    return multivariant_impl(x, M, ldx, variant_ids, w_b, masks, vs, v_stride, axes, V, d_out, d_in, y, ldy, workspace,
+                             workspace_bytes, cuda_stream, true);
+}
+
 pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void *w_b, const uint32_t *mask, const void *v,
                          pd_axis axis, int64_t d_out, int64_t d_in, void *y_dev, void *y_host, void *workspace,
                          size_t workspace_bytes, void *cuda_stream, uint32_t flags) {
@@ -257,16 +311,19 @@ pd_status pd_linear_host(const void *x_host, void *x_dev, int64_t M, const void 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * d_in * sizeof(__half), cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return PD_ERR_CUDA;
-    const pd_status st = pd_linear_ex(x_dev, M, d_in, w_b, mask, v, axis, d_out, d_in, y_dev, d_out, workspace, workspace_bytes,
-                                      cuda_stream, flags);
+    const pd_status st = linear_impl(x_dev, M, d_in, w_b, mask, v, axis, d_out, d_in, y_dev, d_out, workspace, workspace_bytes,
+                                     cuda_stream, flags, false);
     if (st != PD_OK) return st;
     return cuda_ok(cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * d_out * sizeof(__half), cudaMemcpyDeviceToHost, stream));
 }
 
-pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
-                                 const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes,
-                                 int32_t V, int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace,
-                                 size_t workspace_bytes, void *cuda_stream) {
+}  // extern "C"
+
+namespace {
+pd_status multivariant_impl(const void *x, int64_t M, int64_t ldx, const int32_t *variant_ids, const void *w_b,
+                            const uint32_t *masks, const void *vs, int64_t v_stride, const uint8_t *axes, int32_t V,
+                            int64_t d_out, int64_t d_in, void *y, int64_t ldy, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream, bool bf16) {
     pd_status st = check_matrix_args(x, M, ldx, w_b, d_out, d_in, y, ldy);
     if (st != PD_OK) return st;
     if (!variant_ids || !masks || !vs || !axes || V <= 0) return PD_ERR_INVALID_ARG;
@@ -293,7 +350,7 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
     if (M <= kMvDecodeMaxTokens && d_in % 128 == 0)
         // a decode batch: one launch that streams W_b once and applies every variant's mask to its few rows
         return launch_mv_decode(xh, static_cast<int>(M), ldx, variant_ids, static_cast<const __half *>(w_b), masks, mask_words, vh,
-                                v_stride, col_bits, V, d_out, d_in, static_cast<__half *>(y), ldy, base + kStatusBytes, status, stream);
+                                v_stride, col_bits, V, d_out, d_in, static_cast<__half *>(y), ldy, base + kStatusBytes, status, bf16, stream);
     if (M > kGemvMaxTokens && d_in >= 64) {
         // more than one decode chunk: sort the rows by variant, gather them, one grouped tensor-core launch
         unsigned char *p = base + kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256);
@@ -306,20 +363,27 @@ pd_status pd_linear_multivariant(const void *x, int64_t M, int64_t ldx, const in
         return launch_gemm_grouped(x_sorted, M, static_cast<const __half *>(w_b), masks, mask_words, vh, v_stride, col_bits,
                                    V, d_out, d_in, static_cast<__half *>(y), ldy, tile_table, n_token_tiles,
                                    static_cast<int>(M / grouped_token_tile_for(M, V, d_out) + V + 2), grouped_token_tile_for(M, V, d_out), row_index, status,
-                                   stream);
+                                   bf16, stream);
     }
     st = launch_group_rows(variant_ids, static_cast<int>(M), V, offsets, row_index, status, nullptr, nullptr, 0, nullptr, 0, 0,
                            nullptr, stream);
     if (st != PD_OK) return st;
+    GemvScratch scratch;
+    scratch.status = status;
+    scratch.weights_resident = false;
+    scratch.bf16 = bf16;
     for (int g = 0; g <= V; ++g) {
         const bool base_only = (g == V);
         st = launch_gemv(xh, 0, ldx, static_cast<const __half *>(w_b), base_only ? nullptr : masks + g * mask_words,
                          base_only ? nullptr : vh + g * v_stride, base_only ? PD_AXIS_ROW : axes[g], d_out, d_in,
-                         static_cast<__half *>(y), ldy, row_index, offsets, g, nullptr, stream);
+                         static_cast<__half *>(y), ldy, row_index, offsets, g, &scratch, stream);
         if (st != PD_OK) return st;
     }
     return PD_OK;
 }
+}  // namespace
+
+extern "C" {
 
 pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream) {
     if (!workspace || !aligned256(workspace) || limit_cycles <= 0 || limit_cycles > 100000000) return PD_ERR_INVALID_ARG;

@@ -61,21 +61,24 @@ __device__ __forceinline__ void latch_error(uint32_t *status, uint32_t code, uin
 }
 
 // --- launchers implemented in the .cu files (all enqueue on `stream`, none synchronises) ---
+// Weights and activations are 16-bit values passed as __half pointers; `bf16` says that the bits are bfloat16
+// (the scale vectors are binary16 either way).
 size_t pack_scratch_bytes(int64_t d_out, int64_t d_in);  // the sums; zero on entry, zero again on return
 pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
-                      __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream);
+                      __half *v_row, __half *v_col, unsigned long long *sums, bool bf16, cudaStream_t stream);
 pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
-                       int64_t d_in, __half *w_hat, cudaStream_t stream);
+                       int64_t d_in, __half *w_hat, bool bf16, cudaStream_t stream);
 
 // What the decode kernels need from the caller's workspace.
 struct GemvScratch {
     uint32_t *status;        // device status words
     bool weights_resident;   // PD_LINEAR_WEIGHTS_RESIDENT: the weight stream may start before the previous kernel has finished
+    bool bf16;               // x, W_b and y are bfloat16
 };
 
 // M <= 16 tokens (mask == nullptr: base weights only).  With group_offsets != nullptr the tokens are
 // rows row_index[group_offsets[group] .. group_offsets[group+1]) of x / y (any count, read on the device).
-// scratch may be nullptr (then the register-fed kernel runs); it is required for nothing else.
+// scratch carries the status words and the call's switches.
 pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
                       const int *row_index, const int *group_offsets, int group, const GemvScratch *scratch,
@@ -84,7 +87,7 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
 // M > 16 tokens on the tcgen05 tensor cores (needs d_in % 8 == 0; tails in M, d_out and d_in are handled).
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      uint32_t *status, cudaStream_t stream);
+                      uint32_t *status, bool bf16, cudaStream_t stream);
 
 // Multi-variant prefill: x_sorted holds the token rows in bucket order (contiguous, pitch d_in); token tile
 // i of tile_table is {variant (V = base only), first sorted row, rows (<= token_tile), 0}; token_tile is 64, 128
@@ -104,7 +107,7 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
-                              uint32_t *status, cudaStream_t stream);
+                              uint32_t *status, bool bf16, cudaStream_t stream);
 
 // Multi-variant decode: at most kMvDecodeMaxTokens token rows, d_in a multiple of 128.  One launch, one pass over
 // W_b; the kernel buckets the rows by variant id itself (ids outside [-1, V) latch PD_ERR_BAD_VARIANT).
@@ -113,7 +116,7 @@ size_t mv_decode_scratch_bytes(int64_t M, int32_t V, int64_t d_in);  // x and co
 pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *ids, const __half *w_b, const uint32_t *masks,
                            int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits, int V,
                            int64_t d_out, int64_t d_in, __half *y, int64_t ldy, unsigned char *scratch, uint32_t *status,
-                           cudaStream_t stream);
+                           bool bf16, cudaStream_t stream);
 
 // Stable bucket sort of token rows by variant id: offsets[g] .. offsets[g+1] index row_index for
 // variant g (g = 0..V-1), offsets[V] .. offsets[V+1] the rows with id -1.  Other ids latch an error.

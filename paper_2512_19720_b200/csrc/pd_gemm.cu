@@ -65,6 +65,7 @@ struct GemmArgs {
     int V;
     int y_vec_ok;  // y is 16-byte aligned and ldy a multiple of 8: rows can be written with 16-byte stores
     int token_tile;  // pair kernel, one variant: tokens per tile (64, 128 or 256)
+    int bf16;        // host side only: which instantiation to launch
 };
 
 struct Tile {
@@ -161,6 +162,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     return d;
 }
 
+// Instruction descriptor of tcgen05.mma kind::f16 without the shape fields: fp32 accumulator (bit 4), and the
+// format of A and B (bits 7..9 and 10..12): 0 = binary16, 1 = bfloat16 -- both operands always have the same type.
+template <bool BF16>
+constexpr uint32_t kIdescBase = (1u << 4) | (BF16 ? ((1u << 7) | (1u << 10)) : 0u);
+
 template <int BN>
 struct SmemLayout {
     static constexpr int kWBytes = BM * BK * 2;   // 16 KB
@@ -180,7 +186,7 @@ struct SmemLayout {
 
 // One row of a W_hat tile: 64 columns = 8 pieces of 16 bytes read from the 128-byte-swizzled W_b tile, +-v added
 // per mask bit (word0 = columns 0..31, word1 = columns 32..63), packed two fp16 per register in column order.
-template <bool DELTA, bool COL>
+template <bool BF16, bool DELTA, bool COL>
 __device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsigned char *wt, const unsigned char *vs, int r,
                                                 uint32_t vrow, uint32_t word0, uint32_t word1) {
 #pragma unroll
@@ -192,6 +198,10 @@ __device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsig
             if (COL) {
                 const uint4 t4 = *reinterpret_cast<const uint4 *>(vs + 16 * c);
                 vv[0] = t4.x, vv[1] = t4.y, vv[2] = t4.z, vv[3] = t4.w;
+                if (BF16) {  // the scales arrive as binary16: one rounding to the weights' type
+#pragma unroll
+                    for (int pr = 0; pr < 4; ++pr) vv[pr] = Elem<BF16>::scale_pair2(vv[pr]);
+                }
             }
             // the piece's 8 sign bits are byte c & 3 of its word.  b * 0x8001 puts bit i at i and i + 15, so a left
             // shift by 15 - 2 pr brings bit 2 pr to bit 15 and bit 2 pr + 1 to bit 31: the signs of halves 2 pr (low)
@@ -199,7 +209,7 @@ __device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsig
             const uint32_t sp = prmt(c < 4 ? word0 : word1, 0u, 0x4440u | static_cast<uint32_t>(c & 3)) * 0x8001u;
 #pragma unroll
             for (int pr = 0; pr < 4; ++pr)
-                out[4 * c + pr] = hadd2_u32(wp[pr], lop3_andn_xor(sp << (15 - 2 * pr), 0x80008000u, vv[pr]));
+                out[4 * c + pr] = Elem<BF16>::add2(wp[pr], lop3_andn_xor(sp << (15 - 2 * pr), 0x80008000u, vv[pr]));
         } else {  // base only: the tile goes to tensor memory unchanged
 #pragma unroll
             for (int pr = 0; pr < 4; ++pr) out[4 * c + pr] = wp[pr];
@@ -207,7 +217,7 @@ __device__ __forceinline__ void build_w_hat_row(uint32_t (&out)[32], const unsig
     }
 }
 
-template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
+template <bool BF16, int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = SmemLayout<BN>;
@@ -295,7 +305,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 // MMA N = the tile's tokens rounded up to 16 (the whole token box in the plain mode)
                 const Tile ti = get_tile<AXIS, HAS_DELTA, GROUPED, BN>(a, tile, n_tt);
                 const int n_mma = GROUPED ? ((ti.count + 15) & ~15) : BN;
-                const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+                const uint32_t idesc = kIdescBase<BF16> | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
                 const uint32_t b = tcount % kAccBufs;
                 if (!(ok = mbar_wait(acc_empty + b, ((tcount / kAccBufs) & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
@@ -353,7 +363,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                     tcgen05_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        *reinterpret_cast<__half *>(stage_out + (c0 + j) * 256 + row_l * 2) = __float2half_rn(__uint_as_float(r[j]));
+                        *reinterpret_cast<unsigned short *>(stage_out + (c0 + j) * 256 + row_l * 2) = Elem<BF16>::from_float(__uint_as_float(r[j]));
                 }
                 if (hf == n_half - 1) {  // every column of the accumulator has been read
                     tcgen05_fence_before();
@@ -398,8 +408,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             const bool row_ok = o < a.d_out;
             uint32_t vrow = 0;
             if (delta && !col && row_ok) {
-                const uint32_t hv = *reinterpret_cast<const unsigned short *>(ti.v + o);
-                vrow = hv | (hv << 16);
+                vrow = Elem<BF16>::scale_pair(*reinterpret_cast<const unsigned short *>(ti.v + o));
             }
             const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
             auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
@@ -426,9 +435,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 uint32_t out[32];
                 // specialised bodies: with the variant known only at run time (grouped mode) a single body with
                 // the tests inside the unrolled loop spilled registers and ran four times slower
-                if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[0], word[1]);
-                else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[0], word[1]);
-                else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                if (!delta) build_w_hat_row<BF16, false, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                else if (col) build_w_hat_row<BF16, true, true>(out, wt, vs, r, vrow, word[0], word[1]);
+                else build_w_hat_row<BF16, true, false>(out, wt, vs, r, vrow, word[0], word[1]);
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + sa, ((my_it / kASlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
                 tcgen05_fence_after();
                 tcgen05_st_32x32b_x32(a_taddr + sa * 32, out);
@@ -592,7 +601,7 @@ __device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, i
     return t;
 }
 
-template <int AXIS, bool HAS_DELTA, bool GROUPED>
+template <bool BF16, int AXIS, bool HAS_DELTA, bool GROUPED>
 __global__ void __launch_bounds__(pair_threads(GROUPED), 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmArgs a) {
     using L = PairLayout;
@@ -679,7 +688,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             bool ok = true;
             for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++tcount) {
                 const int n_mma = 2 * tile_of(tile).half;
-                const uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
+                const uint32_t idesc = kIdescBase<BF16> | (static_cast<uint32_t>(n_mma >> 3) << 17) | (static_cast<uint32_t>(256 >> 4) << 24);
                 if (!(ok = mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag, a.status, 2))) break;
                 tcgen05_fence_after();
                 for (int ks = 0; ks < a.k_steps; ks += 2, it += 2) {
@@ -741,7 +750,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     tcgen05_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        *reinterpret_cast<__half *>(stage_out + (c0 + j) * 256 + row_l * 2) = __float2half_rn(__uint_as_float(r[j]));
+                        *reinterpret_cast<unsigned short *>(stage_out + (c0 + j) * 256 + row_l * 2) = Elem<BF16>::from_float(__uint_as_float(r[j]));
                 }
                 if (hf == n_half - 1) {  // every column of the accumulator has been read
                     tcgen05_fence_before();
@@ -785,8 +794,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const bool row_ok = o < a.d_out;
             uint32_t vrow = 0;
             if (delta && !col && row_ok) {
-                const uint32_t hv = *reinterpret_cast<const unsigned short *>(ti.v + o);
-                vrow = hv | (hv << 16);
+                vrow = Elem<BF16>::scale_pair(*reinterpret_cast<const unsigned short *>(ti.v + o));
             }
             const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
             auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
@@ -809,9 +817,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 const unsigned char *vs = smem + L::kVOffset + s * kVSlotBytes;
                 uint32_t out[32];
                 // specialised bodies: a single body with run-time tests inside the unrolled loop spills
-                if (!delta) build_w_hat_row<false, false>(out, wt, vs, r, vrow, word[0], word[1]);
-                else if (col) build_w_hat_row<true, true>(out, wt, vs, r, vrow, word[0], word[1]);
-                else build_w_hat_row<true, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                if (!delta) build_w_hat_row<BF16, false, false>(out, wt, vs, r, vrow, word[0], word[1]);
+                else if (col) build_w_hat_row<BF16, true, true>(out, wt, vs, r, vrow, word[0], word[1]);
+                else build_w_hat_row<BF16, true, false>(out, wt, vs, r, vrow, word[0], word[1]);
                 const uint32_t pi = my_it >> 1;  // the W_hat slot was last read by pair pi - 4
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + pi % kPairSlots, ((pi / kPairSlots) & 1) ^ 1, abort_flag, a.status, 8)))) break;
                 tcgen05_fence_after();
@@ -857,9 +865,9 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, in
                        CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
-pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
-    auto kernel = gemm_kernel<AXIS, HAS_DELTA, GROUPED, BN>;
+template <bool BF16, int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
+pd_status launch_one_t(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    auto kernel = gemm_kernel<BF16, AXIS, HAS_DELTA, GROUPED, BN>;
     constexpr int smem = SmemLayout<BN>::kTotal;
     static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
     if (!ensure_dynamic_smem(kernel, smem, configured)) return PD_ERR_CUDA;
@@ -872,10 +880,16 @@ pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArg
 
 namespace {
 
+template <int AXIS, bool HAS_DELTA, bool GROUPED, int BN>
+pd_status launch_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    return args.bf16 ? launch_one_t<true, AXIS, HAS_DELTA, GROUPED, BN>(mw, mx, args, grid, stream)
+                     : launch_one_t<false, AXIS, HAS_DELTA, GROUPED, BN>(mw, mx, args, grid, stream);
+}
+
 template <int BN>
 pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                          int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                         cudaStream_t stream) {
+                         bool bf16, cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, BN)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -890,6 +904,7 @@ pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *
     args.tiles_n = static_cast<int>((M + BN - 1) / BN);
     args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
     args.status = status;
+    args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = args.tiles_m * args.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
@@ -902,9 +917,9 @@ pd_status launch_gemm_bn(const __half *x, int64_t M, int64_t ldx, const __half *
 
 namespace {
 
-template <int AXIS, bool HAS_DELTA, bool GROUPED>
-pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
-    auto kernel = gemm_pair_kernel<AXIS, HAS_DELTA, GROUPED>;
+template <bool BF16, int AXIS, bool HAS_DELTA, bool GROUPED>
+pd_status launch_pair_one_t(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    auto kernel = gemm_pair_kernel<BF16, AXIS, HAS_DELTA, GROUPED>;
     constexpr int smem = PairLayout::kTotal;
     static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
     if (!ensure_dynamic_smem(kernel, smem, configured)) return PD_ERR_CUDA;
@@ -924,10 +939,16 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const Ge
     return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mx, args));
 }
 
+template <int AXIS, bool HAS_DELTA, bool GROUPED>
+pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const GemmArgs &args, int grid, cudaStream_t stream) {
+    return args.bf16 ? launch_pair_one_t<true, AXIS, HAS_DELTA, GROUPED>(mw, mx, args, grid, stream)
+                     : launch_pair_one_t<false, AXIS, HAS_DELTA, GROUPED>(mw, mx, args, grid, stream);
+}
+
 // Tiles of 256 rows x 256 tokens on pairs of CTAs.
 pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                            int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, int token_tile, uint32_t *status,
-                           cudaStream_t stream) {
+                           bool bf16, cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, 128)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -943,6 +964,7 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.token_tile = token_tile;
     args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;  // even: the MMA thread works on pairs of k steps
     args.status = status;
+    args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
     const int pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
@@ -956,7 +978,7 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
                                    int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                                    int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                                    const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
-                                   cudaStream_t stream) {
+                                   bool bf16, cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, 128)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -971,6 +993,7 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
     args.tiles_n = 0;
     args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;
     args.status = status;
+    args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     args.tile_table = tile_table;
     args.n_token_tiles = n_token_tiles;
@@ -988,7 +1011,7 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
 
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      uint32_t *status, cudaStream_t stream) {
+                      uint32_t *status, bool bf16, cudaStream_t stream) {
     const int sms = sm_count();
     if (gemm_pair_enabled() && d_out >= 256) {
         // CTA pairs, tiles of 256 rows x token_tile tokens.  A pair of k steps costs the issuing thread about 1250
@@ -1004,7 +1027,7 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
             const int64_t cost = ((units + pairs - 1) / pairs) * per;
             if (best_tt_cost < 0 || cost <= best_tt_cost) best_tt = tt, best_tt_cost = cost;
         }
-        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, best_tt, status, stream);
+        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, best_tt, status, bf16, stream);
     }
     // One CTA per tile (fewer than 256 output rows).  256 tokens per tile amortise the W_hat transform best, but with
     // few tokens that leaves most SMs without
@@ -1019,9 +1042,9 @@ pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b
         const int64_t cost = ((tiles + sms - 1) / sms) * (2 * bn > 400 ? 2 * bn : 400);
         if (best_cost < 0 || cost <= best_cost) best = bn, best_cost = cost;
     }
-    if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
-    if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
-    return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, stream);
+    if (best == 256) return launch_gemm_bn<256>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, bf16, stream);
+    if (best == 128) return launch_gemm_bn<128>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, bf16, stream);
+    return launch_gemm_bn<64>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, bf16, stream);
 }
 
 namespace {
@@ -1031,7 +1054,7 @@ pd_status launch_gemm_grouped_bn(const __half *x_sorted, int64_t M, const __half
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, const int *row_index, uint32_t *status,
-                              cudaStream_t stream) {
+                              bool bf16, cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x_sorted, M, d_in, d_in, BN)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -1046,6 +1069,7 @@ pd_status launch_gemm_grouped_bn(const __half *x_sorted, int64_t M, const __half
     args.tiles_n = 0;
     args.k_steps = static_cast<int>((d_in + BK - 1) / BK);
     args.status = status;
+    args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
     args.tile_table = tile_table;
     args.n_token_tiles = n_token_tiles;
@@ -1065,13 +1089,13 @@ pd_status launch_gemm_grouped(const __half *x_sorted, int64_t M, const __half *w
                               int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits,
                               int V, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, const int4 *tile_table,
                               const int *n_token_tiles, int max_token_tiles, int token_tile, const int *row_index,
-                              uint32_t *status, cudaStream_t stream) {
+                              uint32_t *status, bool bf16, cudaStream_t stream) {
     if (token_tile == 256 && gemm_pair_enabled() && d_out >= 256)
         return launch_gemm_pair_grouped(x_sorted, M, w_b, masks, mask_stride, vs, v_stride, col_axis_bits, V, d_out, d_in, y, ldy,
-                                        tile_table, n_token_tiles, max_token_tiles, row_index, status, stream);
+                                        tile_table, n_token_tiles, max_token_tiles, row_index, status, bf16, stream);
 #define PD_GROUPED(BN)                                                                                                     \
     return launch_gemm_grouped_bn<BN>(x_sorted, M, w_b, masks, mask_stride, vs, v_stride, col_axis_bits, V, d_out, d_in, y, \
-                                      ldy, tile_table, n_token_tiles, max_token_tiles, row_index, status, stream)
+                                      ldy, tile_table, n_token_tiles, max_token_tiles, row_index, status, bf16, stream)
     if (token_tile == 64) PD_GROUPED(64);
     if (token_tile == 128) PD_GROUPED(128);
     PD_GROUPED(256);

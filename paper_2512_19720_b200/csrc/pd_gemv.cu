@@ -7,14 +7,6 @@
 namespace pd {
 namespace {
 
-__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 // arguments of the generic kernel
 struct GemvArgs {
     const __half *x;
@@ -114,7 +106,7 @@ __device__ __forceinline__ void load_xfrag(XFrag &f, const StreamArgs &a, int k0
     }
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
+template <bool BF16, int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
 __global__ void __maxnreg__(stream_three_per_sm(KS, STAGES) ? 72 : 96)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_m, const StreamArgs a) {
     extern __shared__ unsigned char smem_raw[];
@@ -190,11 +182,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         uint32_t mag[kTiles];  // |B operand| of the delta MMA as a half2: (s, s) for the row axis, (1, 1) for the col axis
 #pragma unroll
         for (int j = 0; j < kTiles; ++j) {
-            mag[j] = 0x3C003C00u;
-            if (HAS_DELTA && AXIS == PD_AXIS_ROW) {
-                const uint32_t h = *reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1));
-                mag[j] = h | (h << 16);
-            }
+            mag[j] = Elem<BF16>::kOnePair;
+            if (HAS_DELTA && AXIS == PD_AXIS_ROW)
+                mag[j] = Elem<BF16>::scale_pair(*reinterpret_cast<const unsigned short *>(a.v + min(row0 + 8 * j + g, a.d_out - 1)));
         }
         // items: (step s, block bb of this warp), k0 = s*kStep + (kItems*warp + bb)*64; x fragments one item ahead
         // (two ahead for up to 8 tokens, where the registers allow it: the loads come from L2, ~1 us away under load)
@@ -231,7 +221,13 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     // |B operand| of the delta MMA for the four half2 pairs of this piece: v[k] itself (col axis),
                     // read from the stage (all lanes with the same t read the same 16 bytes: a broadcast)
                     uint4 vv = make_uint4(0, 0, 0, 0);
-                    if (kCol) vv = *reinterpret_cast<const uint4 *>(stage + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
+                    if (kCol) {
+                        vv = *reinterpret_cast<const uint4 *>(stage + kStV + (blk * 64 + 8 * (t + 4 * c)) * 2);
+                        if (BF16) {  // the scales arrive as binary16: one rounding to the weights' type
+                            vv.x = Elem<BF16>::scale_pair2(vv.x), vv.y = Elem<BF16>::scale_pair2(vv.y);
+                            vv.z = Elem<BF16>::scale_pair2(vv.z), vv.w = Elem<BF16>::scale_pair2(vv.w);
+                        }
+                    }
                     if (M16) {
     #pragma unroll
                         for (int j = 0; j < kTiles; ++j) {
@@ -245,13 +241,13 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 const uint32_t pm1 = lop3_andn_xor(sp << 13, 0x80008000u, kCol ? vv.y : mag[j]);
                                 const uint32_t pm2 = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
                                 const uint32_t pm3 = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
-                                // W_hat = W_b +- v in fp16, as the merge and the prefill path form it: one MMA per
+                                // W_hat = W_b +- v in the weights' 16-bit type, as the merge and the prefill path form it: one MMA per
                                 // 16 columns instead of one for W_b and one for the signs
-                                w.x = hadd2_u32(w.x, pm0), w.y = hadd2_u32(w.y, pm1);
-                                w.z = hadd2_u32(w.z, pm2), w.w = hadd2_u32(w.w, pm3);
+                                w.x = Elem<BF16>::add2(w.x, pm0), w.y = Elem<BF16>::add2(w.y, pm1);
+                                w.z = Elem<BF16>::add2(w.z, pm2), w.w = Elem<BF16>::add2(w.w, pm3);
                             }
-                            mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-                            mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+                            Elem<BF16>::mma16816(acc[j], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+                            Elem<BF16>::mma16816(acc[j], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
                         }
                     } else {
                         // up to 8 tokens: the 16 rows are the MMA's M and the tokens its N, so one MMA does what two
@@ -269,14 +265,14 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                                 pm[j][2] = lop3_andn_xor(sp << 11, 0x80008000u, kCol ? vv.z : mag[j]);
                                 pm[j][3] = lop3_andn_xor(sp << 9, 0x80008000u, kCol ? vv.w : mag[j]);
                             }
-                            w0.x = hadd2_u32(w0.x, pm[0][0]), w0.y = hadd2_u32(w0.y, pm[0][1]);
-                            w0.z = hadd2_u32(w0.z, pm[0][2]), w0.w = hadd2_u32(w0.w, pm[0][3]);
-                            w1.x = hadd2_u32(w1.x, pm[1][0]), w1.y = hadd2_u32(w1.y, pm[1][1]);
-                            w1.z = hadd2_u32(w1.z, pm[1][2]), w1.w = hadd2_u32(w1.w, pm[1][3]);
+                            w0.x = Elem<BF16>::add2(w0.x, pm[0][0]), w0.y = Elem<BF16>::add2(w0.y, pm[0][1]);
+                            w0.z = Elem<BF16>::add2(w0.z, pm[0][2]), w0.w = Elem<BF16>::add2(w0.w, pm[0][3]);
+                            w1.x = Elem<BF16>::add2(w1.x, pm[1][0]), w1.y = Elem<BF16>::add2(w1.y, pm[1][1]);
+                            w1.z = Elem<BF16>::add2(w1.z, pm[1][2]), w1.w = Elem<BF16>::add2(w1.w, pm[1][3]);
                         }
                         // the two pieces of a block go to accumulators of their own: two short chains of dependent MMAs
-                        mma16816(acc[c], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
-                        mma16816(acc[c], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
+                        Elem<BF16>::mma16816(acc[c], w0.x, w1.x, w0.y, w1.y, xa.x, xa.y);
+                        Elem<BF16>::mma16816(acc[c], w0.z, w1.z, w0.w, w1.w, xa.z, xa.w);
                     }
                 }
             }
@@ -326,7 +322,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 float sum = 0.f;
 #pragma unroll
                 for (int w = 0; w < kStreamConsumers; ++w) sum += red[(w * 16 + tok) * R + ol];
-                if (tok < a.M && row0 + ol < a.d_out) a.y[static_cast<size_t>(tok) * a.ldy + row0 + ol] = __float2half_rn(sum);
+                if (tok < a.M && row0 + ol < a.d_out)
+                    reinterpret_cast<unsigned short *>(a.y)[static_cast<size_t>(tok) * a.ldy + row0 + ol] = Elem<BF16>::from_float(sum);
             }
         }
     }
@@ -334,8 +331,9 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 
 // Any d_in that is a multiple of 32 (the tensor path above needs a multiple of 128): one warp per
 // output row, plain fp32 FMAs, shuffle reduction.  Correctness path for odd shapes, not tuned.
-template <int AXIS>
+template <bool BF16, int AXIS>
 __global__ void __launch_bounds__(256) gemv_generic_kernel(const GemvArgs a) {
+    const unsigned short *w_bits = reinterpret_cast<const unsigned short *>(a.w_b), *x_bits = reinterpret_cast<const unsigned short *>(a.x);
     const int lane = threadIdx.x & 31;
     const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (o >= a.d_out) return;
@@ -356,14 +354,14 @@ __global__ void __launch_bounds__(256) gemv_generic_kernel(const GemvArgs a) {
         const uint32_t word = a.mask ? a.mask[static_cast<size_t>(o) * words + w] : 0u;
         for (int b = 0; b < 32; ++b) {
             const int k = 32 * w + b;
-            const float wv = __half2float(a.w_b[static_cast<size_t>(o) * a.d_in + k]);
+            const float wv = Elem<BF16>::to_float(w_bits[static_cast<size_t>(o) * a.d_in + k]);
             float sg = ((word >> b) & 1u) ? 1.f : -1.f;
             if (AXIS == PD_AXIS_COL && a.mask) sg *= __half2float(a.v[k]);
 #pragma unroll
             for (int m = 0; m < 16; ++m) {
                 if (m < M) {
                     const int xr = tok_rows ? tok_rows[tok0 + m] : tok0 + m;
-                    const float xv = __half2float(a.x[static_cast<size_t>(xr) * a.ldx + k]);
+                    const float xv = Elem<BF16>::to_float(x_bits[static_cast<size_t>(xr) * a.ldx + k]);
                     base[m] = fmaf(xv, wv, base[m]);
                     delta[m] = fmaf(xv, sg, delta[m]);
                 }
@@ -378,16 +376,16 @@ __global__ void __launch_bounds__(256) gemv_generic_kernel(const GemvArgs a) {
 #pragma unroll
             for (int sft = 16; sft > 0; sft >>= 1) val += __shfl_xor_sync(0xffffffffu, val, sft);
             const int yr = tok_rows ? tok_rows[tok0 + m] : tok0 + m;
-            if (lane == 0) a.y[static_cast<size_t>(yr) * a.ldy + o] = __float2half_rn(val);
+            if (lane == 0) reinterpret_cast<unsigned short *>(a.y)[static_cast<size_t>(yr) * a.ldy + o] = Elem<BF16>::from_float(val);
         }
     }
   }
 }
 
-template <int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
+template <bool BF16, int AXIS, bool HAS_DELTA, bool M16, int KS, int STAGES>
 pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, const StreamArgs &args, int grid,
                                 cudaStream_t stream) {
-    auto kernel = gemv_stream_kernel<AXIS, HAS_DELTA, M16, KS, STAGES>;
+    auto kernel = gemv_stream_kernel<BF16, AXIS, HAS_DELTA, M16, KS, STAGES>;
     constexpr int kStreamSmem = stream_smem_bytes(KS, STAGES);
     static std::atomic<bool> configured[kMaxDevices];  // per instantiation and device
     if (!ensure_dynamic_smem(kernel, kStreamSmem, configured)) return PD_ERR_CUDA;
@@ -408,7 +406,7 @@ pd_status launch_stream_variant(const CUtensorMap &mw, const CUtensorMap &mm, co
 template <int KS, int STAGES>
 pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                              int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                             bool weights_resident, cudaStream_t stream) {
+                             bool weights_resident, bool bf16, cudaStream_t stream) {
     constexpr int step = KS, R = kStreamRows;
     const bool m16 = M > 8, delta = mask != nullptr;
     CUtensorMap mw, mm;
@@ -430,7 +428,9 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
     // one CTA per tile of R rows: a persistent grid walking several tiles measured slower on the 7B
     // shapes (fewer rings in flight, more registers)
     const int grid = static_cast<int>((d_out + R - 1) / R);
-#define PD_STREAM_CASE(AX, D, W) return launch_stream_variant<AX, D, W, KS, STAGES>(mw, mm, a, grid, stream)
+#define PD_STREAM_CASE(AX, D, W)                                                                      \
+    return bf16 ? launch_stream_variant<true, AX, D, W, KS, STAGES>(mw, mm, a, grid, stream)          \
+                : launch_stream_variant<false, AX, D, W, KS, STAGES>(mw, mm, a, grid, stream)
     if (!delta) {
         if (m16) PD_STREAM_CASE(PD_AXIS_ROW, false, true);
         PD_STREAM_CASE(PD_AXIS_ROW, false, false);
@@ -446,7 +446,7 @@ pd_status launch_stream_rows(const __half *x, int M, int64_t ldx, const __half *
 
 pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
                         int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, uint32_t *status,
-                        bool weights_resident, cudaStream_t stream) {
+                        bool weights_resident, bool bf16, cudaStream_t stream) {
     // Ring depth.  A shorter ring (four steps, 72 KB) lets three CTAs share an SM: the same bytes in flight,
     // but a CTA that is finishing (last step, reduction, store) overlaps two that stream.  It needs a grid that
     // fills three CTAs per SM (smaller grids need six steps per CTA to keep enough in flight) and whose last
@@ -456,8 +456,8 @@ pd_status launch_stream(const __half *x, int M, int64_t ldx, const __half *w_b, 
     const double tiles = static_cast<double>((d_out + kStreamRows - 1) / kStreamRows);
     const double w3 = tiles / (3.0 * sm_count()), w2 = tiles / (2.0 * sm_count());
     const bool three = w3 >= 1.0 && w3 / ceil(w3) >= w2 / ceil(w2) - 0.1;
-    if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, stream);
-    return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, stream);
+    if (three) return launch_stream_rows<512, 4>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, bf16, stream);
+    return launch_stream_rows<512, 6>(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, status, weights_resident, bf16, stream);
 }
 
 }  // namespace
@@ -468,7 +468,7 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       cudaStream_t stream) {
     // plain calls on TMA-friendly shapes stream the weights through shared memory
     if (ws != nullptr && group_offsets == nullptr && d_in % 128 == 0)
-        return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, ws->weights_resident, stream);
+        return launch_stream(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, ws->status, ws->weights_resident, ws->bf16, stream);
     GemvArgs args;
     args.x = x;
     args.w_b = w_b;
@@ -485,10 +485,14 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
     args.group = group;
     const int rows_per_cta = 8;
     const unsigned grid = static_cast<unsigned>((d_out + rows_per_cta - 1) / rows_per_cta);
-    if (axis == PD_AXIS_ROW)
-        gemv_generic_kernel<PD_AXIS_ROW><<<grid, 256, 0, stream>>>(args);
-    else
-        gemv_generic_kernel<PD_AXIS_COL><<<grid, 256, 0, stream>>>(args);
+    const bool bf16 = ws != nullptr && ws->bf16;
+    if (axis == PD_AXIS_ROW) {
+        if (bf16) gemv_generic_kernel<true, PD_AXIS_ROW><<<grid, 256, 0, stream>>>(args);
+        else gemv_generic_kernel<false, PD_AXIS_ROW><<<grid, 256, 0, stream>>>(args);
+    } else {
+        if (bf16) gemv_generic_kernel<true, PD_AXIS_COL><<<grid, 256, 0, stream>>>(args);
+        else gemv_generic_kernel<false, PD_AXIS_COL><<<grid, 256, 0, stream>>>(args);
+    }
     count_launch();
     return cuda_ok(cudaGetLastError());
 }

@@ -151,13 +151,6 @@ __device__ __forceinline__ void mv_sort_rows(MvSort &so, const MvArgs &a, bool r
     __syncthreads();
 }
 
-__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -191,6 +184,7 @@ __device__ __forceinline__ void mv_grid_launch_dependents() { asm volatile("grid
 // (chunk c of a 32-column block holds, for t = 0..3, the pairs (2t, 2t+16), (2t+8, 2t+24), (2t+1, 2t+17),
 // (2t+9, 2t+25) for c = 0..3), and the step's scales of every col-axis variant as pairs
 // {(2t, 2t+16), (2t+1, 2t+17), (2t+8, 2t+24), (2t+9, 2t+25)} per (block, t).
+template <bool BF16>
 __global__ void __launch_bounds__(kMvPrepThreads) mv_prepare_kernel(const MvArgs a) {
     __shared__ MvSort so;
     mv_grid_launch_dependents();  // the decode kernel may start streaming weights; it waits for this grid before it reads x_pairs
@@ -222,14 +216,16 @@ __global__ void __launch_bounds__(kMvPrepThreads) mv_prepare_kernel(const MvArgs
             if (!((a.col_axis_bits >> var) & 1ull)) continue;
             const uint32_t *vw = reinterpret_cast<const uint32_t *>(a.vs + static_cast<size_t>(var) * a.v_stride + k0 + 32 * blk);
             const uint32_t w0 = __ldg(vw + t), w1 = __ldg(vw + t + 4), w2 = __ldg(vw + t + 8), w3 = __ldg(vw + t + 12);
+            // binary16 scales -> the weights' type (one rounding for bfloat16)
             *reinterpret_cast<uint4 *>(a.v_pairs + (static_cast<size_t>(var) * a.steps_total + s) * 256 + blk * 64 + t * 16) =
-                make_uint4(prmt(w0, w2, 0x5410u), prmt(w0, w2, 0x7632u), prmt(w1, w3, 0x5410u), prmt(w1, w3, 0x7632u));
+                make_uint4(Elem<BF16>::scale_pair2(prmt(w0, w2, 0x5410u)), Elem<BF16>::scale_pair2(prmt(w0, w2, 0x7632u)),
+                           Elem<BF16>::scale_pair2(prmt(w1, w3, 0x5410u)), Elem<BF16>::scale_pair2(prmt(w1, w3, 0x7632u)));
         }
     }
 }
 
 // ANYCOL: some variant of the call scales along d_in (its items read their scale pairs from the stage).
-template <bool ANYCOL>
+template <bool BF16, bool ANYCOL>
 __global__ void __launch_bounds__(kMvThreads, 1)
 mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_m, const MvArgs a) {
     extern __shared__ unsigned char smem_raw[];
@@ -289,13 +285,13 @@ mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         // row-axis scales (v, v) per item and row, ldmatrix row offsets per item and lane
         for (int i = threadIdx.x; i < kMvItems * kMvRows; i += kMvThreads) {
             const int it = i / kMvRows, r = i - it * kMvRows;
-            uint32_t h = 0;  // base-only items, col-axis items and padding: +-0
+            uint32_t pair = 0;  // base-only items, col-axis items and padding: +-0
             if (it < n_it) {
                 const int var = so.item_var[item0 + it];
                 if (var < a.V && !((a.col_axis_bits >> var) & 1ull) && row0 + r < a.d_out)
-                    h = *reinterpret_cast<const unsigned short *>(a.vs + static_cast<size_t>(var) * a.v_stride + row0 + r);
+                    pair = Elem<BF16>::scale_pair(*reinterpret_cast<const unsigned short *>(a.vs + static_cast<size_t>(var) * a.v_stride + row0 + r));
             }
-            mag2[i] = h | (h << 16);
+            mag2[i] = pair;
         }
         for (int i = threadIdx.x; i < kMvItems * 32; i += kMvThreads) {
             const int it = min(i >> 5, n_it - 1), l = i & 31;
@@ -422,9 +418,9 @@ mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             if (ANYCOL) vp[j] = lds128(stage + voff + 3 * j * 256 + blk * 64);
                         }
 #pragma unroll
-                        for (int j = 0; j < kMvMine; ++j) mma16816(acc[j], ab[0][0], ab[0][1], ab[0][2], ab[0][3], xb[j][0], xb[j][1]);
+                        for (int j = 0; j < kMvMine; ++j) Elem<BF16>::mma16816(acc[j], ab[0][0], ab[0][1], ab[0][2], ab[0][3], xb[j][0], xb[j][1]);
 #pragma unroll
-                        for (int j = 0; j < kMvMine; ++j) mma16816(acc[j], ab[1][0], ab[1][1], ab[1][2], ab[1][3], xb[j][2], xb[j][3]);
+                        for (int j = 0; j < kMvMine; ++j) Elem<BF16>::mma16816(acc[j], ab[1][0], ab[1][1], ab[1][2], ab[1][3], xb[j][2], xb[j][3]);
                         // +-v from the mask bits: a set bit keeps +v, a clear bit flips the sign
 #pragma unroll
                         for (int j = 0; j < kMvMine; ++j) {
@@ -433,7 +429,7 @@ mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             const uint32_t a3 = m[j] * mul3, b3 = m8[j] * mul3;  // bits 2t+9, 2t+25 on bits 15, 31
                             const uint32_t s0 = lop3_andn_xor(a3 << 9, 0x80008000u, q0), s2 = lop3_andn_xor(a3 << 1, 0x80008000u, q2);
                             const uint32_t u0 = lop3_andn_xor(b3 << 9, 0x80008000u, r0), u2 = lop3_andn_xor(b3 << 1, 0x80008000u, r2);
-                            mma16816(acc[j], s0, u0, s2, u2, xb[j][0], xb[j][1]);
+                            Elem<BF16>::mma16816(acc[j], s0, u0, s2, u2, xb[j][0], xb[j][1]);
                         }
 #pragma unroll
                         for (int j = 0; j < kMvMine; ++j) {
@@ -442,7 +438,7 @@ mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             const uint32_t a3 = m[j] * mul3, b3 = m8[j] * mul3;
                             const uint32_t s1 = lop3_andn_xor(a3 << 8, 0x80008000u, q1), s3 = lop3_andn_xor(a3, 0x80008000u, q3);
                             const uint32_t u1 = lop3_andn_xor(b3 << 8, 0x80008000u, r1), u3 = lop3_andn_xor(b3, 0x80008000u, r3);
-                            mma16816(acc[j], s1, u1, s3, u3, xb[j][2], xb[j][3]);
+                            Elem<BF16>::mma16816(acc[j], s1, u1, s3, u3, xb[j][2], xb[j][3]);
                         }
                     }
                 }
@@ -491,8 +487,9 @@ mv_decode_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 }
                 const int o = row0 + 2 * rp;
                 __half *dst = a.y + static_cast<size_t>(so.tok[so.item_first[item0 + it] + j]) * a.ldy + o;
-                if (o < a.d_out) dst[0] = __float2half_rn(sum.x);
-                if (o + 1 < a.d_out) dst[1] = __float2half_rn(sum.y);
+                unsigned short *out = reinterpret_cast<unsigned short *>(dst);
+                if (o < a.d_out) out[0] = Elem<BF16>::from_float(sum.x);
+                if (o + 1 < a.d_out) out[1] = Elem<BF16>::from_float(sum.y);
             }
         }
         cluster.sync();  // nobody refills the ring (next pass) or leaves while another rank still reads its sums
@@ -524,7 +521,7 @@ size_t mv_decode_scratch_bytes(int64_t M, int32_t V, int64_t d_in) {
 pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *ids, const __half *w_b, const uint32_t *masks,
                            int64_t mask_stride, const __half *vs, int64_t v_stride, unsigned long long col_axis_bits, int V,
                            int64_t d_out, int64_t d_in, __half *y, int64_t ldy, unsigned char *scratch, uint32_t *status,
-                           cudaStream_t stream) {
+                           bool bf16, cudaStream_t stream) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return PD_ERR_CUDA;
     CUtensorMap mw, mm;
@@ -559,7 +556,8 @@ pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *i
     a.x_pairs = scratch;
     a.v_pairs = scratch + round_up(static_cast<size_t>(d_in) * 2 * a.m_pad, 256);
     a.status = status;
-    mv_prepare_kernel<<<a.steps_total, kMvPrepThreads, 0, stream>>>(a);
+    if (bf16) mv_prepare_kernel<true><<<a.steps_total, kMvPrepThreads, 0, stream>>>(a);
+    else mv_prepare_kernel<false><<<a.steps_total, kMvPrepThreads, 0, stream>>>(a);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return PD_ERR_CUDA;
     // column split: the cluster size (<= 8) whose grid fills the SMs best, counting a fixed cost of about three
@@ -573,11 +571,12 @@ pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *i
         const double cost = waves * ((a.steps_total + ks - 1) / ks + 3.0);
         if (ks == 1 || cost < best_cost) best = ks, best_cost = cost;
     }
-    static std::atomic<bool> configured[2][kMaxDevices];
+    static std::atomic<bool> configured[4][kMaxDevices];
     const bool any_col = col_axis_bits != 0;
-    if (!(any_col ? ensure_dynamic_smem(mv_decode_kernel<true>, kMvSmemBytes, configured[1])
-                  : ensure_dynamic_smem(mv_decode_kernel<false>, kMvSmemBytes, configured[0])))
-        return PD_ERR_CUDA;
+    void (*kernel)(CUtensorMap, CUtensorMap, MvArgs) =
+        bf16 ? (any_col ? mv_decode_kernel<true, true> : mv_decode_kernel<true, false>)
+             : (any_col ? mv_decode_kernel<false, true> : mv_decode_kernel<false, false>);
+    if (!ensure_dynamic_smem(kernel, kMvSmemBytes, configured[(bf16 ? 2 : 0) + (any_col ? 1 : 0)])) return PD_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(best), static_cast<unsigned>(row_groups));
     cfg.blockDim = dim3(kMvThreads);
@@ -593,8 +592,7 @@ pd_status launch_mv_decode(const __half *x, int M, int64_t ldx, const int32_t *i
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     count_launch();
-    return cuda_ok(any_col ? cudaLaunchKernelEx(&cfg, mv_decode_kernel<true>, mw, mm, a)
-                           : cudaLaunchKernelEx(&cfg, mv_decode_kernel<false>, mw, mm, a));
+    return cuda_ok(cudaLaunchKernelEx(&cfg, kernel, mw, mm, a));
 }
 
 }  // namespace pd

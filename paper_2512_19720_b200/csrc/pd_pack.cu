@@ -7,7 +7,7 @@
 // lanes form one 32-bit mask word.
 #include <climits>
 
-#include "pd_common.cuh"
+#include "pd_ptx.cuh"
 
 namespace pd {
 
@@ -45,13 +45,13 @@ __device__ __forceinline__ void stg_stream(uint4 *p, uint4 v) {
                  : "memory");
 }
 
-__device__ __forceinline__ __half2 as_half2(uint32_t u) { return *reinterpret_cast<__half2 *>(&u); }
-
-// Signed value of a binary16 in units of 2^-24 (every finite binary16 is an integer number of them).
-__device__ __forceinline__ long long half_units(uint32_t h) {
-    const uint32_t e = (h >> 10) & 31u, m = h & 1023u;
-    const long long mag = e ? (static_cast<long long>(m | 1024u) << (e - 1u)) : static_cast<long long>(m);
-    return (h & 0x8000u) ? -mag : mag;
+// floor(|a - b| * 2^24) for two finite values of at most 2^28 in magnitude: the fp64 difference is taken with
+// rounding toward zero, which cuts |a - b| down to a grid finer than 2^-24 and so never crosses a multiple of
+// 2^-24; the product with 2^24 is exact and the conversion rounds down.  (binary16 differences are multiples of
+// 2^-24 already: nothing is cut.)
+__device__ __forceinline__ unsigned long long abs_diff_units(float a, float b) {
+    const double d = fabs(__dsub_rz(static_cast<double>(a), static_cast<double>(b)));
+    return __double2ull_rd(d * 16777216.0);
 }
 
 // mean = (sum * 2^-24) / n with one fp64 division, then one rounding to binary16
@@ -64,7 +64,7 @@ __device__ __forceinline__ unsigned short mean_to_half(unsigned long long sum, i
 
 // One row of a tile, any position: bounds-checked, exact 64-bit fixed point for every magnitude.  Used for tiles that
 // hang over the matrix edge and for the rare tiles that hold a |dW| >= 0.5.
-template <bool ROW, bool COL>
+template <bool BF16, bool ROW, bool COL>
 __device__ __forceinline__ void pack_row_exact(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int o, int col0,
                                                int d_out, int d_in, uint32_t *__restrict__ mask,
                                                unsigned long long *__restrict__ row_sum,
@@ -78,14 +78,14 @@ __device__ __forceinline__ void pack_row_exact(const uint4 *__restrict__ w_f, co
         const uint32_t a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-            const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p]));
+            const uint32_t ge = Elem<BF16>::ge_mask(a[p], b[p]);
             bits |= ((ge & 1u) << (2 * p)) | (((ge >> 16) & 1u) << (2 * p + 1));
+            const float2 fa = Elem<BF16>::to_float2(a[p]), fb = Elem<BF16>::to_float2(b[p]);
+            const unsigned long long du[2] = {abs_diff_units(fa.x, fb.x), abs_diff_units(fa.y, fb.y)};
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const long long d = half_units((a[p] >> (16 * h)) & 0xffffu) - half_units((b[p] >> (16 * h)) & 0xffffu);
-                const unsigned long long du = static_cast<unsigned long long>(d < 0 ? -d : d);
-                sum += du;
-                if (COL) atomicAdd(col_sum + col0 + 2 * p + h, du);
+                sum += du[h];
+                if (COL) atomicAdd(col_sum + col0 + 2 * p + h, du[h]);
             }
         }
     }
@@ -114,13 +114,14 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // trips per thread, which a 20 us kernel cannot hide; finishing a band in the CTA that draws its last ticket instead
 // of in a second kernel -- the fence and the ticket's round trip hold the whole CTA for longer than its loads take.)
 //
-// |dW| is summed in units of 2^-24, exactly.  The fp32 difference of two binary16 values is exact and a multiple of
-// 2^-24; an fp32 accumulator that starts at 0.5 and stays below 1 has an ulp of 2^-24, so adding |dW| to it is exact
-// and its bit pattern minus that of 0.5 is the sum in units.  A lane keeps one such accumulator per row (8 addends)
-// and one per column (4 addends).  An accumulator that reaches 1 (or is not finite) fails the check and that row,
-// or that warp's share of the columns, is redone by pack_row_exact in 64-bit integers; so are tiles that hang over
-// the matrix edge.
-template <bool ROW, bool COL>
+// What is summed is floor(|dW| * 2^24) units of 2^-24, exactly (for binary16 inputs |dW| is a whole number of them).
+// The fp32 difference rounded toward zero is |dW| cut down to a grid finer than 2^-24 (exact for binary16); an fp32
+// accumulator that starts at 0.5 and stays below 1 has an ulp of 2^-24, so adding |dW| to it with rounding toward
+// zero adds exactly the whole units of |dW|, and its bit pattern minus that of 0.5 is the sum in units.  A lane keeps
+// one such accumulator per row (8 addends) and one per column (4 addends).  An accumulator that reaches 1 (or is
+// not finite) fails the check and that row, or that warp's share of the columns, is redone by pack_row_exact in
+// 64-bit integers; so are tiles that hang over the matrix edge.
+template <bool BF16, bool ROW, bool COL>
 __global__ void __launch_bounds__(kThreads, 4)
 pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_out, int d_in, int tiles_c,
             uint32_t *__restrict__ mask, unsigned long long *__restrict__ row_sum,
@@ -157,14 +158,14 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
             float rf = 0.5f;
 #pragma unroll
             for (int p = 0; p < 4; ++p) {
-                // bit = (w_f >= w_b): exact on binary16, false for NaN, true for -0 vs +0.  The comparison gives
+                // bit = (w_f >= w_b): an exact comparison, false for NaN, true for -0 vs +0.  The comparison gives
                 // 0xffff per true half; pair p keeps bit 2p of the low half and bit 2p+1 of the high half.
-                const uint32_t ge = __hge2_mask(as_half2(a[p]), as_half2(b[p]));
+                const uint32_t ge = Elem<BF16>::ge_mask(a[p], b[p]);
                 spread |= ge & ((1u << (2 * p)) | (1u << (17 + 2 * p)));
-                const float2 fa = __half22float2(as_half2(a[p])), fb = __half22float2(as_half2(b[p]));
-                const float d0 = fabsf(__fsub_rn(fa.x, fb.x)), d1 = fabsf(__fsub_rn(fa.y, fb.y));
-                if (ROW) rf = __fadd_rn(__fadd_rn(rf, d0), d1);
-                if (COL) cf[2 * p] = __fadd_rn(cf[2 * p], d0), cf[2 * p + 1] = __fadd_rn(cf[2 * p + 1], d1);
+                const float2 fa = Elem<BF16>::to_float2(a[p]), fb = Elem<BF16>::to_float2(b[p]);
+                const float d0 = fabsf(__fsub_rz(fa.x, fb.x)), d1 = fabsf(__fsub_rz(fa.y, fb.y));
+                if (ROW) rf = __fadd_rz(__fadd_rz(rf, d0), d1);
+                if (COL) cf[2 * p] = __fadd_rz(cf[2 * p], d0), cf[2 * p + 1] = __fadd_rz(cf[2 * p + 1], d1);
             }
             uint32_t word = ((spread | (spread >> 16)) & 0xffu) << (8 * (lane & 3));
             word |= __shfl_xor_sync(kFull, word, 1);
@@ -176,7 +177,7 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
                     const uint32_t total = __reduce_add_sync(kFull, rb - kHalfBits);  // <= 32 * 2^23 units
                     if (lane == 0) atomicAdd(row_sum + o, static_cast<unsigned long long>(total));
                 } else {
-                    pack_row_exact<true, false>(w_f, w_b, o, col0, d_out, d_in, mask, row_sum, col_sum, lane);
+                    pack_row_exact<BF16, true, false>(w_f, w_b, o, col0, d_out, d_in, mask, row_sum, col_sum, lane);
                 }
             }
         }
@@ -189,12 +190,12 @@ pack_kernel(const uint4 *__restrict__ w_f, const uint4 *__restrict__ w_b, int d_
                 for (int j = 0; j < 8; ++j) cunits[j] = __float_as_uint(cf[j]) - kHalfBits;
             } else {
                 for (int i = 0; i < kRowsPerWarp; ++i)
-                    pack_row_exact<false, true>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
+                    pack_row_exact<BF16, false, true>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
             }
         }
     } else {
         for (int i = 0; i < kRowsPerWarp; ++i)
-            pack_row_exact<ROW, COL>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
+            pack_row_exact<BF16, ROW, COL>(w_f, w_b, row0 + warp + 8 * i, col0, d_out, d_in, mask, row_sum, col_sum, lane);
     }
     if (COL) {
 #pragma unroll
@@ -227,7 +228,7 @@ __global__ void pack_finalize_kernel(unsigned long long *__restrict__ row_sum, u
     dst[j] = mean_to_half(sum, is_row ? d_in : d_out);
 }
 
-template <int AXIS>
+template <bool BF16, int AXIS>
 __global__ void __launch_bounds__(kThreads)
 merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *__restrict__ v, int d_out, int d_in,
              int tiles_c, uint4 *w_hat) {
@@ -243,7 +244,7 @@ merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *
         const uint32_t u[4] = {vv.x, vv.y, vv.z, vv.w};
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-            const float2 f = __half22float2(as_half2(u[p]));
+            const float2 f = Elem<false>::to_float2(u[p]);  // the scales are binary16
             vf[2 * p] = f.x;
             vf[2 * p + 1] = f.y;
         }
@@ -265,11 +266,10 @@ merge_kernel(const uint4 *w_b, const uint32_t *__restrict__ mask, const __half *
         uint32_t r[4];
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-            const float2 f = __half22float2(as_half2(w[p]));
+            const float2 f = Elem<BF16>::to_float2(w[p]);
             const float s0 = __uint_as_float(__float_as_uint(vf[2 * p]) ^ (((nbits >> (2 * p)) & 1u) << 31));
             const float s1 = __uint_as_float(__float_as_uint(vf[2 * p + 1]) ^ (((nbits >> (2 * p + 1)) & 1u) << 31));
-            const __half2 h = __floats2half2_rn(__fadd_rn(f.x, s0), __fadd_rn(f.y, s1));
-            r[p] = *reinterpret_cast<const uint32_t *>(&h);
+            r[p] = Elem<BF16>::from_float2(__fadd_rn(f.x, s0), __fadd_rn(f.y, s1));  // one fp32 add, one rounding to 16 bits
         }
         stg_stream(w_hat + idx, make_uint4(r[0], r[1], r[2], r[3]));
     }
@@ -283,7 +283,7 @@ size_t pack_scratch_bytes(int64_t d_out, int64_t d_in) {
 
 // scratch: pack_scratch_bytes() bytes, all zero on entry; the call leaves them zero again.
 pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64_t d_in, uint32_t *mask,
-                      __half *v_row, __half *v_col, unsigned long long *sums, cudaStream_t stream) {
+                      __half *v_row, __half *v_col, unsigned long long *sums, bool bf16, cudaStream_t stream) {
     unsigned long long *row_sum = sums, *col_sum = sums + d_out;
     const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
     const int64_t tiles = ((d_out + kPackRows - 1) / kPackRows) * tiles_c;
@@ -291,12 +291,17 @@ pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64
     const unsigned grid = static_cast<unsigned>(tiles);
     const uint4 *a = reinterpret_cast<const uint4 *>(w_f), *b = reinterpret_cast<const uint4 *>(w_b);
     const int n_out = static_cast<int>(d_out), n_in = static_cast<int>(d_in);
-    if (v_row && v_col)
-        pack_kernel<true, true><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    else if (v_row)
-        pack_kernel<true, false><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
-    else
-        pack_kernel<false, true><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum);
+#define PD_PACK(BF, R, C) pack_kernel<BF, R, C><<<grid, kThreads, 0, stream>>>(a, b, n_out, n_in, tiles_c, mask, row_sum, col_sum)
+    if (bf16) {
+        if (v_row && v_col) PD_PACK(true, true, true);
+        else if (v_row) PD_PACK(true, true, false);
+        else PD_PACK(true, false, true);
+    } else {
+        if (v_row && v_col) PD_PACK(false, true, true);
+        else if (v_row) PD_PACK(false, true, false);
+        else PD_PACK(false, false, true);
+    }
+#undef PD_PACK
     if (cudaGetLastError() != cudaSuccess) return PD_ERR_CUDA;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled while the pack kernel runs
@@ -313,16 +318,21 @@ pd_status launch_pack(const __half *w_f, const __half *w_b, int64_t d_out, int64
 }
 
 pd_status launch_merge(const __half *w_b, const uint32_t *mask, const __half *v, int axis, int64_t d_out,
-                       int64_t d_in, __half *w_hat, cudaStream_t stream) {
+                       int64_t d_in, __half *w_hat, bool bf16, cudaStream_t stream) {
     const int tiles_c = static_cast<int>((d_in + kTileCols - 1) / kTileCols);
     const int64_t tiles = ((d_out + kTileRows - 1) / kTileRows) * tiles_c;
     const dim3 grid(static_cast<unsigned>(tiles)), block(kThreads);
     const uint4 *b = reinterpret_cast<const uint4 *>(w_b);
     uint4 *out = reinterpret_cast<uint4 *>(w_hat);
-    if (axis == PD_AXIS_ROW)
-        merge_kernel<PD_AXIS_ROW><<<grid, block, 0, stream>>>(b, mask, v, (int)d_out, (int)d_in, tiles_c, out);
-    else
-        merge_kernel<PD_AXIS_COL><<<grid, block, 0, stream>>>(b, mask, v, (int)d_out, (int)d_in, tiles_c, out);
+#define PD_MERGE(BF, AX) merge_kernel<BF, AX><<<grid, block, 0, stream>>>(b, mask, v, (int)d_out, (int)d_in, tiles_c, out)
+    if (bf16) {
+        if (axis == PD_AXIS_ROW) PD_MERGE(true, PD_AXIS_ROW);
+        else PD_MERGE(true, PD_AXIS_COL);
+    } else {
+        if (axis == PD_AXIS_ROW) PD_MERGE(false, PD_AXIS_ROW);
+        else PD_MERGE(false, PD_AXIS_COL);
+    }
+#undef PD_MERGE
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
@@ -372,6 +382,6 @@ extern "C" pd_status pd_pack_delta_static(const void *w_f, const void *w_b, int6
     if (sums == nullptr) return PD_ERR_CUDA;
     // the array starts zero-filled (device globals do) and every call puts what it used back to zero
     return launch_pack(static_cast<const __half *>(w_f), static_cast<const __half *>(w_b), d_out, d_in, mask,
-                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums,
+                       static_cast<__half *>(v_row), static_cast<__half *>(v_col), sums, false,
                        static_cast<cudaStream_t>(cuda_stream));
 }

@@ -3,6 +3,8 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -111,6 +113,75 @@ __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
     asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
+
+// ------------------------------------------------------------------ the two storage types of weights and activations
+// Elem<false>: IEEE binary16; Elem<true>: bfloat16 (paper, Implementation remarks: the base is kept in BF16).  Values
+// travel as raw bits (one element per unsigned short, two per 32-bit register, the lower index in the lower half).
+// The scale vectors are binary16 in both cases.
+template <bool BF16>
+struct Elem;
+
+template <>
+struct Elem<false> {
+    static constexpr uint32_t kOnePair = 0x3C003C00u;  // (1.0, 1.0)
+    static __device__ __forceinline__ float to_float(unsigned short h) { return __half2float(__ushort_as_half(h)); }
+    static __device__ __forceinline__ float2 to_float2(uint32_t p) { return __half22float2(*reinterpret_cast<const __half2 *>(&p)); }
+    static __device__ __forceinline__ unsigned short from_float(float f) { return __half_as_ushort(__float2half_rn(f)); }
+    static __device__ __forceinline__ uint32_t from_float2(float lo, float hi) {
+        const __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    }
+    static __device__ __forceinline__ uint32_t add2(uint32_t a, uint32_t b) { return hadd2_u32(a, b); }
+    // 0xffff in every half where a >= b (false for NaN, true for -0 against +0)
+    static __device__ __forceinline__ uint32_t ge_mask(uint32_t a, uint32_t b) {
+        return __hge2_mask(*reinterpret_cast<const __half2 *>(&a), *reinterpret_cast<const __half2 *>(&b));
+    }
+    // a binary16 scale as a pair (s, s) of elements, and a pair of binary16 scales as a pair of elements
+    static __device__ __forceinline__ uint32_t scale_pair(unsigned short v) { return static_cast<uint32_t>(v) | (static_cast<uint32_t>(v) << 16); }
+    static __device__ __forceinline__ uint32_t scale_pair2(uint32_t v2) { return v2; }
+    static __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
+
+template <>
+struct Elem<true> {
+    static constexpr uint32_t kOnePair = 0x3F803F80u;
+    static __device__ __forceinline__ float to_float(unsigned short h) { return __uint_as_float(static_cast<uint32_t>(h) << 16); }
+    static __device__ __forceinline__ float2 to_float2(uint32_t p) { return make_float2(__uint_as_float(p << 16), __uint_as_float(p & 0xffff0000u)); }
+    static __device__ __forceinline__ unsigned short from_float(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
+    static __device__ __forceinline__ uint32_t from_float2(float lo, float hi) {
+        uint32_t d;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+        return d;
+    }
+    static __device__ __forceinline__ uint32_t add2(uint32_t a, uint32_t b) {
+        uint32_t d;
+        asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    static __device__ __forceinline__ uint32_t ge_mask(uint32_t a, uint32_t b) {
+        return __hge2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+    }
+    // the scale is rounded to bfloat16 once, to nearest even
+    static __device__ __forceinline__ uint32_t scale_pair(unsigned short v) {
+        const uint32_t b = from_float(__half2float(__ushort_as_half(v)));
+        return b | (b << 16);
+    }
+    static __device__ __forceinline__ uint32_t scale_pair2(uint32_t v2) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&v2));
+        return from_float2(f.x, f.y);
+    }
+    static __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
 
 // ------------------------------------------------------------------ host: tensor maps
 using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

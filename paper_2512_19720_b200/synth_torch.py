@@ -19,7 +19,7 @@ def gen_base(d_out, d_in, seed, device):
 
 
 def gen_finetuned(w_b, seed, sigma=1e-3):
-    """W_f = fp16(W_b + fp16(sigma * s_r[o] * z)), s_r ~ U(0.5, 2) per row."""
+    """W_f = W_b + fp16(sigma * s_r[o] * z) rounded to the dtype of W_b (float16 or bfloat16), s_r ~ U(0.5, 2) per row."""
     d_out, d_in = w_b.shape
     g = _gen(w_b.device, seed * 7919 + 2)
     s_r = 0.5 + 1.5 * torch.rand(d_out, generator=g, device=w_b.device, dtype=torch.float32)
@@ -29,7 +29,7 @@ def gen_finetuned(w_b, seed, sigma=1e-3):
         r1 = min(d_out, r0 + rows)
         z = torch.randn((r1 - r0, d_in), generator=g, device=w_b.device, dtype=torch.float32)
         dw16 = (z * (sigma * s_r[r0:r1])[:, None]).half()
-        w_f[r0:r1] = (w_b[r0:r1].double() + dw16.double()).half()
+        w_f[r0:r1] = (w_b[r0:r1].double() + dw16.double()).to(w_b.dtype)
     return w_f
 
 
