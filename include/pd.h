@@ -176,6 +176,39 @@ pd_status pd_merge(const void *w_b, const uint32_t *mask, const void *v, pd_axis
                    int64_t d_out, int64_t d_in, void *w_hat, void *cuda_stream);
 
 /*
+ * pd_load_merged -- cold start of a fine-tuned variant: apply a saved delta to a resident base, module by module.
+ * Paper: Algorithm "Model-wide application from a saved delta file" (for every projection module take its mask and
+ * scale vector and patch the layer); Implementation remarks (the packed deltas move "in a single operation per
+ * module", non-blocking); the load-time paragraph of the experiments (applying the delta on a resident base against
+ * loading a full checkpoint).
+ *
+ * Every module's artifact is ONE contiguous host buffer: d_out * d_in / 32 mask words, then the scale vector (d_out
+ * or d_in binary16 values), pd_artifact_bytes() in all.  The call queues, for module i, one host-to-device copy of
+ * that buffer into half (i mod 2) of `staging` on copy_stream and one pd_merge on compute_stream; the copy of module
+ * i + 1 overlaps the merge of module i, and a staging half is not overwritten before the merge that reads it has
+ * finished (events order the two streams).  Nothing is synchronised: when compute_stream has drained, every w_hat
+ * holds bf16/fp16( fp32(w_b) +- fp32(v) ) exactly as pd_merge / pd_merge_bf16 would have written it.
+ *
+ *   modules      : HOST array of n descriptors (read during the call only)
+ *   staging      : device, at least 2 * max_i pd_artifact_bytes(module i) rounded up to 256, 256-byte aligned
+ *   copy_stream, compute_stream : two different streams for overlap (the same stream works, without overlap);
+ *                  artifacts in pinned host memory make the copies asynchronous
+ * Errors seen on the host (NULL, bad axis or dtype, d_in not a multiple of 32, short staging) return before anything
+ * is queued.
+ */
+typedef struct {
+    const void *w_b;      /* device: base weights [d_out, d_in] */
+    void *w_hat;          /* device: merged weights [d_out, d_in]; may be w_b itself */
+    const void *artifact; /* HOST: mask words, then scales */
+    int64_t d_out, d_in;
+    int32_t axis;         /* pd_axis */
+    int32_t bf16;         /* 0: weights are binary16, 1: bfloat16 */
+} pd_module;
+size_t pd_artifact_bytes(int64_t d_out, int64_t d_in, pd_axis axis);
+pd_status pd_load_merged(const pd_module *modules, int32_t n, void *staging, size_t staging_bytes,
+                         void *copy_stream, void *compute_stream);
+
+/*
  * BF16 variants -- the same four operations with the base, the fine-tuned weights, the activations and the outputs
  * in bfloat16 (the upper 16 bits of an IEEE binary32, passed as void*); masks, ids and the binary16 scale vectors
  * are unchanged.

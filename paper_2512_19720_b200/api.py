@@ -20,8 +20,15 @@ LIB_PATH = os.path.join(_HERE, "libpd.so")
 
 EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_ex", "pd_linear_multivariant", "pd_merge",
            "pd_workspace_bytes", "pd_device_status", "pd_status_string", "pd_launch_count", "pd_selftest_bounded_wait",
-           "pd_pack_delta_bf16", "pd_merge_bf16", "pd_linear_bf16", "pd_linear_multivariant_bf16"]
+           "pd_pack_delta_bf16", "pd_merge_bf16", "pd_linear_bf16", "pd_linear_multivariant_bf16",
+           "pd_artifact_bytes", "pd_load_merged"]
 LINEAR_WEIGHTS_RESIDENT = 1
+
+
+class PdModule(ctypes.Structure):
+    """pd_module of include/pd.h."""
+    _fields_ = [("w_b", ctypes.c_void_p), ("w_hat", ctypes.c_void_p), ("artifact", ctypes.c_void_p),
+                ("d_out", ctypes.c_int64), ("d_in", ctypes.c_int64), ("axis", ctypes.c_int32), ("bf16", ctypes.c_int32)]
 
 
 class PdError(RuntimeError):
@@ -58,6 +65,10 @@ def _load() -> ctypes.CDLL:
     lib.pd_device_status.restype = ctypes.c_int
     lib.pd_status_string.argtypes = [ctypes.c_int]
     lib.pd_status_string.restype = ctypes.c_char_p
+    lib.pd_artifact_bytes.argtypes = [i64, i64, ctypes.c_int]
+    lib.pd_artifact_bytes.restype = sz
+    lib.pd_load_merged.argtypes = [ctypes.POINTER(PdModule), i32, p, sz, p, p]
+    lib.pd_load_merged.restype = ctypes.c_int
     lib.pd_launch_count.argtypes = []
     lib.pd_launch_count.restype = i64
     for name, proto in (("pd_pack_delta_bf16", lib.pd_pack_delta), ("pd_merge_bf16", lib.pd_merge),
@@ -239,6 +250,34 @@ def pd_merge(w_b, mask, v, axis, w_hat=None):
     assert w_hat.dtype == w_b.dtype
     _check((lib.pd_merge_bf16 if bf16 else lib.pd_merge)(_ptr(w_b), _ptr(mask), _ptr(v), int(axis), d_out, d_in, _ptr(w_hat), _stream()), "pd_merge")
     return w_hat
+
+
+def artifact_bytes(d_out: int, d_in: int, axis: int) -> int:
+    return int(lib.pd_artifact_bytes(d_out, d_in, int(axis)))
+
+
+def make_artifact(mask, v, pin=True):
+    """One contiguous host buffer (uint8): the mask words, then the scales (the layout pd_load_merged copies)."""
+    d_out, words = mask.shape
+    mask_bytes = (d_out * words * 4 + 15) // 16 * 16
+    buf = torch.zeros(mask_bytes + (v.numel() * 2 + 15) // 16 * 16, dtype=torch.uint8)
+    buf[:d_out * words * 4] = mask.detach().cpu().contiguous().view(torch.uint8).reshape(-1)
+    buf[mask_bytes:mask_bytes + v.numel() * 2] = v.detach().cpu().contiguous().view(torch.uint8).reshape(-1)
+    return buf.pin_memory() if pin else buf
+
+
+def pd_load_merged(modules, staging, copy_stream):
+    """modules: sequence of (w_b, w_hat, artifact (host uint8 tensor from make_artifact), axis).  The copies go to
+    copy_stream (a torch.cuda.Stream), the merges to the current stream; nothing is synchronised."""
+    arr = (PdModule * len(modules))()
+    for i, (w_b, w_hat, art, axis) in enumerate(modules):
+        bf16 = _elem(w_b, "w_b")
+        assert w_hat.dtype == w_b.dtype and w_b.is_contiguous() and w_hat.is_contiguous() and not art.is_cuda
+        d_out, d_in = w_b.shape
+        assert art.numel() >= artifact_bytes(d_out, d_in, axis)
+        arr[i] = PdModule(w_b.data_ptr(), w_hat.data_ptr(), art.data_ptr(), d_out, d_in, int(axis), int(bf16))
+    _check(lib.pd_load_merged(arr, len(modules), _ptr(staging), staging.numel() * staging.element_size(),
+                              copy_stream.cuda_stream, _stream()), "pd_load_merged")
 
 
 def pd_selftest_bounded_wait(limit_cycles=100000, workspace=None, device=None):

@@ -385,6 +385,63 @@ pd_status multivariant_impl(const void *x, int64_t M, int64_t ldx, const int32_t
 
 extern "C" {
 
+size_t pd_artifact_bytes(int64_t d_out, int64_t d_in, pd_axis axis) {
+    if (d_out <= 0 || d_in <= 0 || d_in % 32 != 0) return 0;
+    const size_t mask_bytes = static_cast<size_t>(d_out) * static_cast<size_t>(d_in / 32) * 4;
+    return round_up(mask_bytes, 16) + round_up(2 * static_cast<size_t>(axis == PD_AXIS_ROW ? d_out : d_in), 16);
+}
+
+pd_status pd_load_merged(const pd_module *modules, int32_t n, void *staging, size_t staging_bytes, void *copy_stream,
+                         void *compute_stream) {
+    if (!modules || n <= 0 || !staging) return PD_ERR_INVALID_ARG;
+    if (!aligned256(staging)) return PD_ERR_ALIGNMENT;
+    size_t half = 0;
+    for (int i = 0; i < n; ++i) {
+        const pd_module &m = modules[i];
+        if (!m.w_b || !m.w_hat || !m.artifact || m.d_out <= 0 || m.d_in <= 0) return PD_ERR_INVALID_ARG;
+        if ((m.axis != PD_AXIS_ROW && m.axis != PD_AXIS_COL) || (m.bf16 != 0 && m.bf16 != 1)) return PD_ERR_INVALID_ARG;
+        if (m.d_in % 32 != 0 || m.d_out > INT_MAX / 2 || m.d_in > INT_MAX / 2) return PD_ERR_UNSUPPORTED_SHAPE;
+        if (!aligned16(m.w_b) || !aligned16(m.w_hat)) return PD_ERR_ALIGNMENT;
+        const size_t bytes = round_up(pd_artifact_bytes(m.d_out, m.d_in, static_cast<pd_axis>(m.axis)), 256);
+        half = bytes > half ? bytes : half;
+    }
+    if (staging_bytes < 2 * half) return PD_ERR_WORKSPACE;
+    cudaStream_t copy = static_cast<cudaStream_t>(copy_stream), compute = static_cast<cudaStream_t>(compute_stream);
+    cudaEvent_t copied[2] = {nullptr, nullptr}, merged[2] = {nullptr, nullptr}, start = nullptr;
+    pd_status st = PD_OK;
+    for (int b = 0; b < 2 && st == PD_OK; ++b)
+        if (cudaEventCreateWithFlags(&copied[b], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&merged[b], cudaEventDisableTiming) != cudaSuccess)
+            st = PD_ERR_CUDA;
+    if (st == PD_OK && cudaEventCreateWithFlags(&start, cudaEventDisableTiming) != cudaSuccess) st = PD_ERR_CUDA;
+    // the copies may not start before work queued earlier on the compute stream (which may still read the staging
+    // buffer or write the base) has finished
+    if (st == PD_OK && (cudaEventRecord(start, compute) != cudaSuccess || cudaStreamWaitEvent(copy, start, 0) != cudaSuccess))
+        st = PD_ERR_CUDA;
+    for (int i = 0; i < n && st == PD_OK; ++i) {
+        const pd_module &m = modules[i];
+        const int b = i & 1;
+        unsigned char *dst = static_cast<unsigned char *>(staging) + b * half;
+        const size_t mask_bytes = round_up(static_cast<size_t>(m.d_out) * static_cast<size_t>(m.d_in / 32) * 4, 16);
+        if (i >= 2 && cudaStreamWaitEvent(copy, merged[b], 0) != cudaSuccess) st = PD_ERR_CUDA;  // the half is free again
+        if (st == PD_OK && cudaMemcpyAsync(dst, m.artifact, pd_artifact_bytes(m.d_out, m.d_in, static_cast<pd_axis>(m.axis)),
+                                           cudaMemcpyHostToDevice, copy) != cudaSuccess)
+            st = PD_ERR_CUDA;
+        if (st == PD_OK && (cudaEventRecord(copied[b], copy) != cudaSuccess || cudaStreamWaitEvent(compute, copied[b], 0) != cudaSuccess))
+            st = PD_ERR_CUDA;
+        if (st == PD_OK)
+            st = merge_impl(m.w_b, reinterpret_cast<const uint32_t *>(dst), dst + mask_bytes, static_cast<pd_axis>(m.axis), m.d_out,
+                            m.d_in, m.w_hat, compute_stream, m.bf16 != 0);
+        if (st == PD_OK && cudaEventRecord(merged[b], compute) != cudaSuccess) st = PD_ERR_CUDA;
+    }
+    for (int b = 0; b < 2; ++b) {  // destroying an event that is still pending only releases it once it has completed
+        if (copied[b]) cudaEventDestroy(copied[b]);
+        if (merged[b]) cudaEventDestroy(merged[b]);
+    }
+    if (start) cudaEventDestroy(start);
+    return st;
+}
+
 pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream) {
     if (!workspace || !aligned256(workspace) || limit_cycles <= 0 || limit_cycles > 100000000) return PD_ERR_INVALID_ARG;
     bounded_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<uint32_t *>(workspace), limit_cycles);
