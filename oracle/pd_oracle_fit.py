@@ -85,3 +85,34 @@ def adamw_step(v, m1, m2, g, t, lr, b1=0.9, b2=0.999, eps=1e-8, wd=0.01):
         assert a.dtype == np.float64 and a.flags.c_contiguous
     g = np.ascontiguousarray(g, dtype=np.float64)
     _load().pdf_adamw_step(_ptr(v), _ptr(m1), _ptr(m2), _ptr(g), v.shape[0], int(t), lr, b1, b2, eps, wd)
+
+
+def train(x_tr, y_tr, x_val, y_val, w_b, mask, v0, axis, epochs, batch, lr, b1=0.9, b2=0.999, eps=1e-8, wd=0.01, cosine=False):
+    """Algorithm "Train per-row/column scaling vectors via activation matching": for each epoch, for each minibatch
+    (consecutive `batch` tokens of the training cache, the last one possibly shorter): loss, gradient with respect to
+    v only, one AdamW step; with `cosine` the step k = 0 .. T-1 (T = all steps) uses lr * (1 + cos(pi k / T)) / 2.
+    Then the validation loss without gradient.  Returns (v, validation loss)."""
+    v = np.array(v0, dtype=np.float64)
+    m1, m2 = np.zeros_like(v), np.zeros_like(v)
+    m_tr = x_tr.shape[0]
+    total = epochs * ((m_tr + batch - 1) // batch)
+    k = 0
+    for _ in range(epochs):
+        for b0 in range(0, m_tr, batch):
+            _, g = loss_grad(x_tr[b0:b0 + batch], y_tr[b0:b0 + batch], w_b, mask, v, axis)
+            lr_k = lr * 0.5 * (1.0 + np.cos(np.pi * k / total)) if cosine else lr
+            k += 1
+            adamw_step(v, m1, m2, g, k, lr_k, b1, b2, eps, wd)
+    val, _ = loss_grad(x_val, y_val, w_b, mask, v, axis, want_grad=False)
+    return v, val
+
+
+def fit_layer(x_tr, y_tr, x_val, y_val, w_b, mask, v_row0, v_col0, epochs, batch, lr, **kw):
+    """Algorithm "Per-layer compression with Row/Col selection": both variants start from the packed scales and get
+    the same budget; the row variant is kept when E_row <= E_col.  The error compared is the validation loss of the
+    layer's outputs (the paper's training paragraph: "selected by validation MSE on the held-out shard").
+    Returns (axis, v of that axis, (E_row, E_col), (v_row, v_col))."""
+    v_col, e_col = train(x_tr, y_tr, x_val, y_val, w_b, mask, np.asarray(v_col0, dtype=np.float64), AXIS_COL, epochs, batch, lr, **kw)
+    v_row, e_row = train(x_tr, y_tr, x_val, y_val, w_b, mask, np.asarray(v_row0, dtype=np.float64), AXIS_ROW, epochs, batch, lr, **kw)
+    axis = AXIS_ROW if e_row <= e_col else AXIS_COL
+    return axis, (v_row if axis == AXIS_ROW else v_col), (e_row, e_col), (v_row, v_col)

@@ -152,6 +152,46 @@ def check_descent_lowers_the_loss_and_selection_prefers_the_matching_axis():
     assert final[ROW] <= final[COL]
 
 
+def check_training_loop_matches_a_torch_loop():
+    # the loop of the training algorithm against autograd + torch.optim.AdamW + CosineAnnealingLR stepped per minibatch
+    w_b, _, mask, v_row, v_col, x, y = case(12, 64, 40, 7)
+    xv, yv = x[32:], y[32:]
+    b = torch.from_numpy(signs(mask, 64))
+    wt = torch.from_numpy(w_b.astype(np.float64))
+    for axis, cosine in ((ROW, False), (COL, True)):
+        v0 = start_vector(axis, v_row, v_col)
+        v_o, val_o = orc.train(x[:32], y[:32], xv, yv, w_b, mask, v0, axis, epochs=3, batch=12, lr=1e-4, cosine=cosine)
+        p = torch.nn.Parameter(torch.from_numpy(v0.copy()))
+        opt = torch.optim.AdamW([p], lr=1e-4, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01)
+        sched = torch.optim.lr_scheduler.CosineAnnealingLR(opt, T_max=9) if cosine else None
+
+        def forward(xa):
+            s = p[:, None] if axis == ROW else p[None, :]
+            return torch.from_numpy(xa.astype(np.float64)) @ (wt + s * b).T
+
+        for _ in range(3):
+            for b0 in (0, 12, 24):
+                opt.zero_grad()
+                loss = torch.mean((forward(x[b0:min(b0 + 12, 32)]) - torch.from_numpy(y[b0:min(b0 + 12, 32)].astype(np.float64))) ** 2)
+                loss.backward()
+                opt.step()
+                if sched:
+                    sched.step()
+        val_t = torch.mean((forward(xv) - torch.from_numpy(yv.astype(np.float64))) ** 2).item()
+        assert np.allclose(v_o, p.detach().numpy(), rtol=1e-9, atol=1e-15), axis
+        assert abs(val_o - val_t) <= 1e-10 * max(1.0, val_t)
+
+
+def check_selection_keeps_the_lower_validation_loss():
+    w_b, _, mask, v_row, v_col, x, y = case(16, 64, 40, 8)
+    axis, v, (e_row, e_col), (vr, vc) = orc.fit_layer(x[:32], y[:32], x[32:], y[32:], w_b, mask, v_row, v_col, epochs=2, batch=16, lr=1e-4)
+    assert axis == (ROW if e_row <= e_col else COL)
+    assert np.array_equal(v, vr if axis == ROW else vc)
+    for a, vec, e in ((ROW, vr, e_row), (COL, vc, e_col)):
+        again, _ = orc.loss_grad(x[32:], y[32:], w_b, mask, vec, a, want_grad=False)
+        assert again == e
+
+
 CHECKS = [v for k, v in sorted(globals().items()) if k.startswith("check_")]
 
 
