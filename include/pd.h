@@ -55,14 +55,17 @@ typedef enum {
 
 typedef enum {
     PD_AXIS_ROW = 0, /* v has d_out entries, W_hat[o,i] = W_b[o,i] + v[o] * B[o,i] */
-    PD_AXIS_COL = 1  /* v has d_in  entries, W_hat[o,i] = W_b[o,i] + v[i] * B[o,i] */
+    PD_AXIS_COL = 1, /* v has d_in  entries, W_hat[o,i] = W_b[o,i] + v[i] * B[o,i] */
+    PD_AXIS_SCALAR = 2 /* pd_fit_* only: one scale for the whole matrix (the scalar baseline the paper compares with) */
 } pd_axis;
 
 typedef enum {
     PD_OP_PACK = 0,
     PD_OP_LINEAR = 1,
     PD_OP_LINEAR_MULTIVARIANT = 2,
-    PD_OP_MERGE = 3
+    PD_OP_MERGE = 3,
+    PD_OP_FIT = 4,       /* pd_fit_loss_grad: M = tokens of the batch */
+    PD_OP_FIT_LAYER = 5  /* pd_fit_layer: M = max(batch, M_val) */
 } pd_op;
 
 /*
@@ -284,6 +287,62 @@ pd_status pd_device_status(void *workspace, void *cuda_stream);
  * The GPU context stays usable.  workspace: at least 256 bytes, 256-byte aligned, zero-filled.
  */
 pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream);
+
+/*
+ * ---- Fitting the scales by output matching ----
+ * Paper: section "Calibration cache, training, and stacking" (per layer, only v is trained, on cached pairs (X, Y) of
+ * the layer's inputs and the fine-tuned layer's outputs, with L = (1/n) ||Y - Y_hat||_2^2 and AdamW); Algorithm "Train
+ * per-row/column scaling vectors via activation matching"; Algorithm "Per-layer compression with Row/Col selection"
+ * (both axes are trained from the packed scales with the same budget, the lower validation loss wins, row on a tie).
+ * n = M * d_out (the mean over all output entries).  W_b, x, y are fp16; v, gradients and optimiser state are fp32
+ * device arrays; every product runs on the tensor cores with fp32 accumulation, W_b and the sign matrix as separate
+ * operands.  Sizes: d_in a multiple of 32, d_out a multiple of 8, M >= 1; x [M, d_in] and y [M, d_out] contiguous,
+ * x and w_b 16-byte aligned.  All calls enqueue on the stream and return; errors the device latches (a bounded wait
+ * that ran out) are read with pd_device_status(workspace).
+ */
+
+/* mask_t [d_in, ceil(d_out/32)] words: bit (o % 32) of mask_t[i][o / 32] = bit (i % 32) of mask[o][i / 32]; rows past
+ * d_out read as 0.  Needed by the col-axis gradient (a contraction over the output rows); computed once per layer. */
+pd_status pd_transpose_mask(const uint32_t *mask, int64_t d_out, int64_t d_in, uint32_t *mask_t, void *cuda_stream);
+
+/*
+ * pd_fit_loss_grad -- loss of one batch and its gradient with respect to v.
+ *   v      : in, fp32, d_out (ROW), d_in (COL) or 1 (SCALAR) entries
+ *   mask_t : in, from pd_transpose_mask; only read for PD_AXIS_COL with grad != NULL (may be NULL otherwise)
+ *   loss   : out, one fp32 (may be NULL);   grad : out, fp32, as many entries as v (NULL: loss only)
+ *   workspace: pd_workspace_bytes(PD_OP_FIT, M, 0, d_out, d_in), 256-byte aligned, status words zero on first use
+ * Partial sums are added in a fixed order: the same inputs give the same bits on every call.
+ */
+pd_status pd_fit_loss_grad(const void *x, const void *y, int64_t M, const void *w_b, const uint32_t *mask,
+                           const uint32_t *mask_t, const float *v, pd_axis axis, int64_t d_out, int64_t d_in, float *loss,
+                           float *grad, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* AdamW constants (decoupled weight decay; the paper fixes the optimiser and the learning rate, 1e-4, only). */
+typedef struct pd_adamw {
+    float lr, beta1, beta2, eps, weight_decay;
+} pd_adamw;
+
+/* One AdamW step, t = 1, 2, ...:  v *= 1 - lr * wd;  m1 = b1 m1 + (1 - b1) g;  m2 = b2 m2 + (1 - b2) g^2;
+ * v -= lr * (m1 / (1 - b1^t)) / (sqrt(m2 / (1 - b2^t)) + eps).  v, m1, m2, grad: fp32 device arrays of len entries. */
+pd_status pd_fit_adamw_step(float *v, float *m1, float *m2, const float *grad, int64_t len, int64_t t, const pd_adamw *opt,
+                            void *cuda_stream);
+
+/*
+ * pd_fit_layer -- the whole per-layer fit with Row/Col selection.
+ *   x_tr [M_tr, d_in], y_tr [M_tr, d_out] : training cache, walked in minibatches of `batch` tokens (the last one may
+ *                                           be shorter), `epochs` times; batch * d_in must keep x 16-byte aligned
+ *   x_val, y_val [M_val, ...]             : held-out cache; the axis with the lower validation loss is kept
+ *   v_row0 [d_out], v_col0 [d_in]         : fp16 starting scales (pd_pack_delta's v_row and v_col)
+ *   cosine != 0                           : learning rate lr * (1 + cos(pi k / T)) / 2 at step k = 0 .. T-1, T = all steps
+ *   v_out    : out, fp16, max(d_out, d_in) entries: the chosen axis' trained scales in its first entries
+ *   axis_out : out, device int32: PD_AXIS_ROW or PD_AXIS_COL
+ *   val_loss : out, device fp32 [2]: validation loss of the row variant, of the col variant
+ *   workspace: pd_workspace_bytes(PD_OP_FIT_LAYER, max(batch, M_val), 0, d_out, d_in)
+ */
+pd_status pd_fit_layer(const void *x_tr, const void *y_tr, int64_t M_tr, const void *x_val, const void *y_val, int64_t M_val,
+                       const void *w_b, const uint32_t *mask, const void *v_row0, const void *v_col0, int64_t d_out,
+                       int64_t d_in, int32_t epochs, int64_t batch, const pd_adamw *opt, int32_t cosine, void *v_out,
+                       int32_t *axis_out, float *val_loss, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* Human-readable name of a status code; never NULL. */
 const char *pd_status_string(pd_status status);

@@ -13,7 +13,8 @@ import torch
 
 AXIS_ROW = 0
 AXIS_COL = 1
-OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE = 0, 1, 2, 3
+AXIS_SCALAR = 2  # pd_fit_* only
+OP_PACK, OP_LINEAR, OP_LINEAR_MULTIVARIANT, OP_MERGE, OP_FIT, OP_FIT_LAYER = 0, 1, 2, 3, 4, 5
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpd.so")
@@ -21,7 +22,8 @@ LIB_PATH = os.path.join(_HERE, "libpd.so")
 EXPORTS = ["pd_pack_delta", "pd_pack_delta_static", "pd_linear_host", "pd_linear", "pd_linear_ex", "pd_linear_multivariant", "pd_merge",
            "pd_workspace_bytes", "pd_device_status", "pd_status_string", "pd_launch_count", "pd_selftest_bounded_wait",
            "pd_pack_delta_bf16", "pd_merge_bf16", "pd_linear_bf16", "pd_linear_multivariant_bf16",
-           "pd_artifact_bytes", "pd_load_merged"]
+           "pd_artifact_bytes", "pd_load_merged",
+           "pd_transpose_mask", "pd_fit_loss_grad", "pd_fit_adamw_step", "pd_fit_layer"]
 LINEAR_WEIGHTS_RESIDENT = 1
 
 
@@ -29,6 +31,12 @@ class PdModule(ctypes.Structure):
     """pd_module of include/pd.h."""
     _fields_ = [("w_b", ctypes.c_void_p), ("w_hat", ctypes.c_void_p), ("artifact", ctypes.c_void_p),
                 ("d_out", ctypes.c_int64), ("d_in", ctypes.c_int64), ("axis", ctypes.c_int32), ("bf16", ctypes.c_int32)]
+
+
+class PdAdamW(ctypes.Structure):
+    """pd_adamw of include/pd.h."""
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+                ("weight_decay", ctypes.c_float)]
 
 
 class PdError(RuntimeError):
@@ -69,6 +77,14 @@ def _load() -> ctypes.CDLL:
     lib.pd_artifact_bytes.restype = sz
     lib.pd_load_merged.argtypes = [ctypes.POINTER(PdModule), i32, p, sz, p, p]
     lib.pd_load_merged.restype = ctypes.c_int
+    lib.pd_transpose_mask.argtypes = [p, i64, i64, p, p]
+    lib.pd_transpose_mask.restype = ctypes.c_int
+    lib.pd_fit_loss_grad.argtypes = [p, p, i64, p, p, p, p, ctypes.c_int, i64, i64, p, p, p, sz, p]
+    lib.pd_fit_loss_grad.restype = ctypes.c_int
+    lib.pd_fit_adamw_step.argtypes = [p, p, p, p, i64, i64, ctypes.POINTER(PdAdamW), p]
+    lib.pd_fit_adamw_step.restype = ctypes.c_int
+    lib.pd_fit_layer.argtypes = [p, p, i64, p, p, i64, p, p, p, p, i64, i64, i32, i64, ctypes.POINTER(PdAdamW), i32, p, p, p, p, sz, p]
+    lib.pd_fit_layer.restype = ctypes.c_int
     lib.pd_launch_count.argtypes = []
     lib.pd_launch_count.restype = i64
     for name, proto in (("pd_pack_delta_bf16", lib.pd_pack_delta), ("pd_merge_bf16", lib.pd_merge),
@@ -278,6 +294,63 @@ def pd_load_merged(modules, staging, copy_stream):
         arr[i] = PdModule(w_b.data_ptr(), w_hat.data_ptr(), art.data_ptr(), d_out, d_in, int(axis), int(bf16))
     _check(lib.pd_load_merged(arr, len(modules), _ptr(staging), staging.numel() * staging.element_size(),
                               copy_stream.cuda_stream, _stream()), "pd_load_merged")
+
+
+def pd_transpose_mask(mask, d_out, d_in, mask_t=None):
+    """mask_t [d_in, ceil(d_out/32)]: the sign mask with the roles of rows and columns exchanged."""
+    _want(mask, torch.int32, "mask")
+    if mask_t is None:
+        mask_t = torch.empty(d_in, (d_out + 31) // 32, dtype=torch.int32, device=mask.device)
+    _check(lib.pd_transpose_mask(_ptr(mask), d_out, d_in, _ptr(mask_t), _stream()), "pd_transpose_mask")
+    return mask_t
+
+
+def adamw(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01) -> PdAdamW:
+    return PdAdamW(lr, beta1, beta2, eps, weight_decay)
+
+
+def pd_fit_loss_grad(x, y, w_b, mask, v, axis, mask_t=None, want_grad=True, loss=None, grad=None, workspace=None):
+    """Loss of the batch (x, y) and its gradient with respect to the fp32 scales v; returns (loss, grad) device tensors."""
+    _want(x, torch.float16, "x"), _want(y, torch.float16, "y"), _want(w_b, torch.float16, "w_b")
+    _want(mask, torch.int32, "mask"), _want(v, torch.float32, "v")
+    m, d_in = x.shape
+    d_out = w_b.shape[0]
+    if loss is None:
+        loss = torch.empty(1, dtype=torch.float32, device=x.device)
+    if grad is None and want_grad:
+        grad = torch.empty_like(v)
+    need = workspace_bytes(OP_FIT, m, 0, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, x.device)
+    _check(lib.pd_fit_loss_grad(_ptr(x), _ptr(y), m, _ptr(w_b), _ptr(mask), _ptr(mask_t), _ptr(v), int(axis), d_out, d_in,
+                                _ptr(loss), _ptr(grad) if want_grad else None, _ptr(ws), ws.numel(), _stream()), "pd_fit_loss_grad")
+    return loss, grad
+
+
+def pd_fit_adamw_step(v, m1, m2, grad, t, opt: PdAdamW):
+    for name, a in (("v", v), ("m1", m1), ("m2", m2), ("grad", grad)):
+        _want(a, torch.float32, name)
+    _check(lib.pd_fit_adamw_step(_ptr(v), _ptr(m1), _ptr(m2), _ptr(grad), v.numel(), int(t), ctypes.byref(opt), _stream()),
+           "pd_fit_adamw_step")
+
+
+def pd_fit_layer(x_tr, y_tr, x_val, y_val, w_b, mask, v_row0, v_col0, epochs, batch, opt: PdAdamW, cosine=False, workspace=None):
+    """Trains both axis variants and keeps the one with the lower validation loss.
+    Returns (v_out fp16 [max(d_out, d_in)], axis_out int32 [1], val_loss fp32 [2]) as device tensors."""
+    for name, a in (("x_tr", x_tr), ("y_tr", y_tr), ("x_val", x_val), ("y_val", y_val), ("w_b", w_b), ("v_row0", v_row0), ("v_col0", v_col0)):
+        _want(a, torch.float16, name)
+    _want(mask, torch.int32, "mask")
+    d_out, d_in = w_b.shape
+    dev = w_b.device
+    v_out = torch.zeros(max(d_out, d_in), dtype=torch.float16, device=dev)
+    axis_out = torch.zeros(1, dtype=torch.int32, device=dev)
+    val_loss = torch.zeros(2, dtype=torch.float32, device=dev)
+    m_max = max(min(batch, x_tr.shape[0]), x_val.shape[0])
+    need = workspace_bytes(OP_FIT_LAYER, m_max, 0, d_out, d_in)
+    ws = workspace if workspace is not None else _workspace(need, dev)
+    _check(lib.pd_fit_layer(_ptr(x_tr), _ptr(y_tr), x_tr.shape[0], _ptr(x_val), _ptr(y_val), x_val.shape[0], _ptr(w_b), _ptr(mask),
+                            _ptr(v_row0), _ptr(v_col0), d_out, d_in, int(epochs), int(batch), ctypes.byref(opt), int(bool(cosine)),
+                            _ptr(v_out), _ptr(axis_out), _ptr(val_loss), _ptr(ws), ws.numel(), _stream()), "pd_fit_layer")
+    return v_out, axis_out, val_loss
 
 
 def pd_selftest_bounded_wait(limit_cycles=100000, workspace=None, device=None):

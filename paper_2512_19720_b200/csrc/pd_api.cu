@@ -168,6 +168,10 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
                 return kStatusBytes + mv_decode_scratch_bytes(M, V, d_in);
             return kStatusBytes + kOffsetsBytes + round_up(sizeof(int) * static_cast<size_t>(M), 256) +
                    (M > kGemvMaxTokens ? grouped_table_bytes(M, V) + round_up(static_cast<size_t>(M) * d_in * 2, 256) : 0);
+        case PD_OP_FIT:
+            return M > 0 ? kStatusBytes + fit_scratch_bytes(M, d_out, d_in) : 0;
+        case PD_OP_FIT_LAYER:
+            return M > 0 ? kStatusBytes + fit_layer_scratch_bytes(M, M, d_out, d_in) : 0;
         case PD_OP_MERGE:
         default:
             return 0;
@@ -440,6 +444,65 @@ pd_status pd_load_merged(const pd_module *modules, int32_t n, void *staging, siz
     }
     if (start) cudaEventDestroy(start);
     return st;
+}
+
+static pd_status fit_shape_check(int64_t M, int64_t d_out, int64_t d_in) {
+    if (M <= 0 || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || d_out % 8 != 0 || M > (1ll << 30) / 128 * 128 || d_out > (1 << 30) || d_in > (1 << 30)) return PD_ERR_UNSUPPORTED_SHAPE;
+    return PD_OK;
+}
+
+pd_status pd_transpose_mask(const uint32_t *mask, int64_t d_out, int64_t d_in, uint32_t *mask_t, void *cuda_stream) {
+    if (!mask || !mask_t || d_out <= 0 || d_in <= 0) return PD_ERR_INVALID_ARG;
+    if (d_in % 32 != 0 || (d_out + 31) / 32 > 65535) return PD_ERR_UNSUPPORTED_SHAPE;
+    return launch_transpose_mask(mask, d_out, d_in, mask_t, static_cast<cudaStream_t>(cuda_stream));
+}
+
+pd_status pd_fit_loss_grad(const void *x, const void *y, int64_t M, const void *w_b, const uint32_t *mask,
+                           const uint32_t *mask_t, const float *v, pd_axis axis, int64_t d_out, int64_t d_in, float *loss,
+                           float *grad, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!x || !y || !w_b || !mask || !v) return PD_ERR_INVALID_ARG;
+    if (axis != PD_AXIS_ROW && axis != PD_AXIS_COL && axis != PD_AXIS_SCALAR) return PD_ERR_INVALID_ARG;
+    if (axis == PD_AXIS_COL && grad && !mask_t) return PD_ERR_INVALID_ARG;
+    const pd_status shape = fit_shape_check(M, d_out, d_in);
+    if (shape != PD_OK) return shape;
+    if (!aligned16(x) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_FIT, M, 0, d_out, d_in)) return PD_ERR_WORKSPACE;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    return launch_fit_loss_grad(static_cast<const __half *>(x), static_cast<const __half *>(y), M, static_cast<const __half *>(w_b), mask,
+                                mask_t, v, axis, d_out, d_in, loss, grad, ws + kStatusBytes, reinterpret_cast<uint32_t *>(ws),
+                                static_cast<cudaStream_t>(cuda_stream));
+}
+
+pd_status pd_fit_adamw_step(float *v, float *m1, float *m2, const float *grad, int64_t len, int64_t t, const pd_adamw *opt,
+                            void *cuda_stream) {
+    if (!v || !m1 || !m2 || !grad || !opt || len <= 0 || t <= 0 || len > (1ll << 31) - 256) return PD_ERR_INVALID_ARG;
+    return launch_fit_adamw(v, m1, m2, grad, len, t, opt->lr, opt->beta1, opt->beta2, opt->eps, opt->weight_decay, nullptr,
+                            static_cast<cudaStream_t>(cuda_stream));
+}
+
+pd_status pd_fit_layer(const void *x_tr, const void *y_tr, int64_t M_tr, const void *x_val, const void *y_val, int64_t M_val,
+                       const void *w_b, const uint32_t *mask, const void *v_row0, const void *v_col0, int64_t d_out,
+                       int64_t d_in, int32_t epochs, int64_t batch, const pd_adamw *opt, int32_t cosine, void *v_out,
+                       int32_t *axis_out, float *val_loss, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!x_tr || !y_tr || !x_val || !y_val || !w_b || !mask || !v_row0 || !v_col0 || !opt || !v_out || !axis_out || !val_loss)
+        return PD_ERR_INVALID_ARG;
+    if (epochs < 0 || batch <= 0) return PD_ERR_INVALID_ARG;
+    pd_status shape = fit_shape_check(M_tr, d_out, d_in);
+    if (shape == PD_OK) shape = fit_shape_check(M_val, d_out, d_in);
+    if (shape != PD_OK) return shape;
+    if ((d_out + 31) / 32 > 65535) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(x_tr) || !aligned16(x_val) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
+    if (batch > M_tr) batch = M_tr;
+    const int64_t m_max = batch > M_val ? batch : M_val;
+    if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_FIT_LAYER, m_max, 0, d_out, d_in))
+        return PD_ERR_WORKSPACE;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    return launch_fit_layer(static_cast<const __half *>(x_tr), static_cast<const __half *>(y_tr), M_tr, static_cast<const __half *>(x_val),
+                            static_cast<const __half *>(y_val), M_val, static_cast<const __half *>(w_b), mask,
+                            static_cast<const __half *>(v_row0), static_cast<const __half *>(v_col0), d_out, d_in, epochs, batch, *opt,
+                            cosine, static_cast<__half *>(v_out), axis_out, val_loss, ws + kStatusBytes,
+                            reinterpret_cast<uint32_t *>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
 pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *cuda_stream) {

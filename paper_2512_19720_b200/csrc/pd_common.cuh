@@ -126,4 +126,19 @@ pd_status launch_group_rows(const int32_t *ids, int M, int V, int *offsets, int 
                             int4 *tile_table, int *n_token_tiles, int token_tile, const __half *x, int64_t ldx,
                             int64_t d_in, __half *x_sorted, cudaStream_t stream);
 
+
+// Scale fitting (pd_fit.cu).  v, gradients and optimiser state are fp32; axis may also be PD_AXIS_SCALAR.
+size_t fit_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in);
+size_t fit_layer_scratch_bytes(int64_t m_batch, int64_t m_val, int64_t d_out, int64_t d_in);
+pd_status launch_transpose_mask(const uint32_t *mask, int64_t d_out, int64_t d_in, uint32_t *mask_t, cudaStream_t stream);
+pd_status launch_fit_loss_grad(const __half *x, const __half *y, int64_t M, const __half *w_b, const uint32_t *mask,
+                               const uint32_t *mask_t, const float *v, int axis, int64_t d_out, int64_t d_in, float *loss,
+                               float *grad, unsigned char *scratch, uint32_t *status, cudaStream_t stream);
+pd_status launch_fit_adamw(float *v, float *m1, float *m2, const float *g, int64_t len, int64_t t, float lr, float b1, float b2,
+                           float eps, float wd, __half *v16, cudaStream_t stream);
+pd_status launch_fit_layer(const __half *x_tr, const __half *y_tr, int64_t m_tr, const __half *x_val, const __half *y_val,
+                           int64_t m_val, const __half *w_b, const uint32_t *mask, const __half *v_row0, const __half *v_col0,
+                           int64_t d_out, int64_t d_in, int epochs, int64_t batch, const pd_adamw &opt, int cosine, __half *v_out,
+                           int32_t *axis_out, float *val_loss, unsigned char *scratch, uint32_t *status, cudaStream_t stream);
+
 }  // namespace pd

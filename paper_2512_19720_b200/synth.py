@@ -131,3 +131,9 @@ def sample_rows(m: int, n_random: int = 64, seed: int = 4000) -> np.ndarray:
     base = [r for r in range(m) if (r % 128) in (0, 1, 127)]
     extra = _rng(seed, 99).integers(0, m, size=n_random).tolist()
     return np.array(sorted(set(base + extra)), dtype=np.int64)
+
+
+def gen_teacher_outputs(x: np.ndarray, w_f: np.ndarray) -> np.ndarray:
+    """Calibration targets of one layer: the fine-tuned layer's outputs for the inputs x, stored as float16
+    (a dense layer's forward pass in fp64 -- input data for the scale fit, not part of the method)."""
+    return (x.astype(np.float64) @ w_f.astype(np.float64).T).astype(np.float16)
