@@ -11,6 +11,8 @@ A step is one pass of the whole path, all through the C ABI, inputs resident in 
                    per row; the same with one id per 512-row sequence; both batch sizes with mixed axes
     merge          pd_merge on the 7 linears, row and col
     bf16_*         pack, decode (M in {1, 4, 16}), prefill (M = 2048) and merge with bfloat16 weights and activations
+    fit_*          one training step of the scales per linear (pd_fit_loss_grad + pd_fit_adamw_step) on 2048 calibration
+                   tokens, row axis and col axis
   single 1024 x 1024 layer
     c1_*           pd_linear at M = 1 and 16 over 128 rotated copies (weights from HBM) and on one copy (L2-resident)
   Llama-70B-shaped block, 80 layers streamed through one set of per-layer buffers
@@ -48,6 +50,7 @@ DECODE_M = (1, 4, 16)
 PREFILL_M = (256, 2048, 8192)
 N_VARIANTS = 16
 MULTI_M = (64, 64 + 4 * 512)
+FIT_M = 2048  # calibration tokens per training step of the scale fit
 C1_COPIES = 128
 ROW, COL = 0, 1
 # ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the captures summarised in profiles/;
@@ -197,6 +200,16 @@ def oracle_other_ops():
             axes = np.zeros(N_VARIANTS, dtype=np.uint8)
             dt = _timed(lambda: orc.linear_multivariant(x, ids, w_b, masks, vs, axes), 1)
             out[f"multivariant_m64_v16_{tag}_GBps"] = round(multi_bytes(64, d_out, d_in) / dt / 1e9, 3)
+    # one loss + gradient evaluation of the scale fit on 4 calibration tokens (4096x4096), both axes
+    from oracle import pd_oracle_fit as orc_fit
+    w_b = synth.gen_base(4096, 4096, 0)
+    w_f = synth.gen_finetuned(w_b, 1000)
+    mask, v_row, v_col = orc.pack(w_f, w_b)
+    x = synth.gen_x(4, 4096, 2004)
+    y = synth.gen_teacher_outputs(x, w_f)
+    for axis, v, mult in ((ROW, v_row, 2), (COL, v_col, 3)):
+        dt = _timed(lambda: orc_fit.loss_grad(x, y, w_b, mask, v.astype("float64"), axis), 1)
+        out[f"fit_{'row' if axis == ROW else 'col'}_4096x4096_GFLOPps (4 tokens)"] = round(mult * 2.0 * 4 * 4096 * 4096 / dt / 1e9, 3)
     out["cores"] = orc.threads()
     return out
 
@@ -321,6 +334,17 @@ def run_ours(args):
         mask, v_row, v_col = api.pd_pack_delta(w_f, w_b)
         bf_layers.append(dict(name=name, d_out=d_out, d_in=d_in, w_b=w_b, w_f=w_f, mask=mask, v=(v_row, v_col),
                               w_hat=torch.empty_like(w_b)))
+    # scale fitting: teacher outputs of the fine-tuned layers for 2048 calibration tokens, fp32 scales and optimiser state
+    fit = []
+    for L in layers:
+        xs = x_all[L["d_in"]][:FIT_M]
+        st = {}
+        for axis, v0 in ((ROW, L["v"][0]), (COL, L["v"][1])):
+            v = v0.float().contiguous()
+            st[axis] = dict(v=v, m1=torch.zeros_like(v), m2=torch.zeros_like(v), g=torch.zeros_like(v))
+        fit.append(dict(L=L, y=(xs @ L["w_f"].T).contiguous(), mask_t=api.pd_transpose_mask(L["mask"], L["d_out"], L["d_in"]),
+                        st=st, loss=torch.zeros(1, device=dev)))
+    fit_opt = api.adamw(lr=1e-4)
     bf_x = {d_in: x_all[d_in][:2048].bfloat16() for d_in in x_all}
     bf_y = {d_out: torch.empty((2048, d_out), dtype=torch.bfloat16, device=dev) for d_out in y_all}
     torch.cuda.synchronize()
@@ -360,6 +384,15 @@ def run_ours(args):
         for axis in (ROW, COL):
             for L in bf_layers:
                 api.pd_merge(L["w_b"], L["mask"], L["v"][axis], axis, w_hat=L["w_hat"])
+
+    def run_fit(axis):
+        # one training step per layer: loss, gradient and AdamW update (step 1 of the bias correction every time, so
+        # that replays do the same arithmetic; the updates still move v)
+        for F in fit:
+            L, st = F["L"], F["st"][axis]
+            api.pd_fit_loss_grad(x_all[L["d_in"]][:FIT_M], F["y"], L["w_b"], L["mask"], st["v"], axis, mask_t=F["mask_t"],
+                                 loss=F["loss"], grad=st["g"])
+            api.pd_fit_adamw_step(st["v"], st["m1"], st["m2"], st["g"], 1, fit_opt)
 
     def run_c1(m, rotated):
         for c in range(C1_COPIES):
@@ -414,6 +447,8 @@ def run_ours(args):
         "gemv_stream_kernel<bf16>")
     add("bf16_prefill_m2048", lambda: bf_linear((2048,), False), 2 * flops(2048), "TFLOP/s", 14, "gemm_pair_kernel<bf16>")
     add("bf16_merge", bf_merge, S["merge"]["work"], "GB/s", 14, "merge_kernel<bf16>")
+    add("fit_row_m2048", lambda: run_fit(ROW), 2 * 2 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<row> (two tcgen05 accumulators)")
+    add("fit_col_m2048", lambda: run_fit(COL), 3 * 2 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<col forward>, <col backward>")
     for m in (1, 16):
         for rotated in (True, False):
             add(f"c1_m{m}_{'rotated' if rotated else 'resident'}", lambda m=m, r=rotated: run_c1(m, r),

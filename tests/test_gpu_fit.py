@@ -149,3 +149,46 @@ def test_fit_argument_errors():
     with pytest.raises(api.PdError) as e:
         api.pd_fit_loss_grad(d[0], d[1], d[2], d[3], dev(v_row.astype(np.float32)), 3)
     assert e.value.code == 1
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d_out,d_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_full_size_layers_on_sampled_rows(d_out, d_in):
+    # 7B-shaped layers with 2048 calibration tokens.  The row gradient of output row o depends on that row only, so the
+    # oracle evaluates a sample of rows (its loss over those rows is the mean of their squared residuals); the col
+    # gradient needs every row and is checked on the first 32 tokens.
+    from paper_2512_19720_b200 import api, synth_torch
+    m = 2048
+    dev0 = torch.device("cuda")
+    w_b = synth_torch.gen_base(d_out, d_in, 7, dev0)
+    w_f = synth_torch.gen_finetuned(w_b, 1007, 3e-3)
+    mask, v_row, v_col = api.pd_pack_delta(w_f, w_b)
+    x = synth_torch.gen_x(m, d_in, 2007, dev0)
+    y = torch.empty(m, d_out, dtype=torch.float16, device=dev0)
+    for r0 in range(0, d_out, 2048):  # teacher outputs in fp64 blocks, rounded once to fp16
+        y[:, r0:r0 + 2048] = (x.double() @ w_f[r0:r0 + 2048].double().T).half()
+    mask_t = api.pd_transpose_mask(mask, d_out, d_in)
+    rows = np.sort(synth.sample_rows(d_out, 24, seed=d_out + d_in))
+    h = lambda t: t.cpu().numpy()
+    v32 = (v_row.float() * 0.6).contiguous()
+    loss, grad = api.pd_fit_loss_grad(x, y, w_b, mask, v32, ROW)
+    assert api.pd_device_status() == 0
+    loss_o, grad_o = orc.loss_grad(h(x), h(y[:, rows].contiguous()), h(w_b[rows].contiguous()), h(mask[rows].contiguous()).view(np.uint32),
+                                   h(v32[rows]).astype(np.float64), ROW)
+    g = h(grad)[rows].astype(np.float64) * (d_out / len(rows))  # the oracle's n counts the sampled rows only
+    assert np.all(np.abs(g - grad_o) <= 3e-3 * np.abs(grad_o) + 3e-3 * np.sqrt(np.mean(grad_o ** 2)))
+    # whole-matrix properties: the scalar gradient is the sum of the row gradients at a constant vector, same loss
+    c = torch.full((d_out,), float(v32.mean()), device=dev0)
+    loss_r, grad_r = api.pd_fit_loss_grad(x, y, w_b, mask, c, ROW)
+    loss_s, grad_s = api.pd_fit_loss_grad(x, y, w_b, mask, c[:1].contiguous(), SCALAR)
+    assert loss_s.item() == loss_r.item()
+    assert abs(grad_s.item() - grad_r.double().sum().item()) <= 1e-5 * grad_r.double().abs().sum().item()
+    # col axis on 32 tokens against the oracle in full
+    mc = 32
+    vc32 = (v_col.float() * 0.6).contiguous()
+    loss_c, grad_c = api.pd_fit_loss_grad(x[:mc], y[:mc], w_b, mask, vc32, COL, mask_t=mask_t)
+    assert api.pd_device_status() == 0
+    loss_co, grad_co = orc.loss_grad(h(x[:mc]), h(y[:mc]), h(w_b), h(mask).view(np.uint32), h(vc32).astype(np.float64), COL)
+    assert abs(loss_c.item() - loss_co) <= 2e-3 * loss_co
+    gc = h(grad_c).astype(np.float64)
+    assert np.all(np.abs(gc - grad_co) <= 3e-3 * np.abs(grad_co) + 3e-3 * np.sqrt(np.mean(grad_co ** 2)))
