@@ -160,8 +160,8 @@ size_t pd_workspace_bytes(int op, int64_t M, int32_t V, int64_t d_out, int64_t d
     switch (op) {
         case PD_OP_PACK:
             return kStatusBytes + pack_scratch_bytes(d_out, d_in);
-        case PD_OP_LINEAR:
-            return kStatusBytes;
+        case PD_OP_LINEAR:  // + the fp32 partial sums when few tokens make the tensor-core path split its k loop
+            return kStatusBytes + ((M > kGemvMaxTokens && d_in >= 64 && d_out > 0) ? gemm_partial_bytes(M, d_out, d_in) : 0);
         case PD_OP_LINEAR_MULTIVARIANT:
             if (M <= 0 || V <= 0) return kStatusBytes + kOffsetsBytes;
             if (M <= kMvDecodeMaxTokens && d_in % 128 == 0)  // decode batches: x (and col-axis scales) re-laid out
@@ -238,7 +238,8 @@ pd_status linear_impl(const void *x, int64_t M, int64_t ldx, const void *w_b, co
     __half *yh = static_cast<__half *>(y);
     if (M > kGemvMaxTokens && d_in >= 64)  // narrower layers would need a TMA box wider than the matrix
         return launch_gemm(xh, M, ldx, static_cast<const __half *>(w_b), mask, static_cast<const __half *>(v), axis,
-                           d_out, d_in, yh, ldy, static_cast<uint32_t *>(workspace), bf16, stream);
+                           d_out, d_in, yh, ldy, reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + kStatusBytes),
+                           static_cast<uint32_t *>(workspace), bf16, stream);
     GemvScratch scratch;
     scratch.status = static_cast<uint32_t *>(workspace);
     scratch.weights_resident = (flags & PD_LINEAR_WEIGHTS_RESIDENT) != 0;

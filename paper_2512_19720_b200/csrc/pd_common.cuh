@@ -85,9 +85,13 @@ pd_status launch_gemv(const __half *x, int M, int64_t ldx, const __half *w_b, co
                       cudaStream_t stream);
 
 // M > 16 tokens on the tcgen05 tensor cores (needs d_in % 8 == 0; tails in M, d_out and d_in are handled).
+// With few tokens the k loop is dealt to several tiles (split-K): `partial` then holds gemm_partial_bytes() of fp32
+// partial sums (0 bytes when the call does not split; nullptr is fine then).
+size_t gemm_partial_bytes(int64_t M, int64_t d_out, int64_t d_in);
+int pair_split_steps(int64_t d_in, int splits);
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      uint32_t *status, bool bf16, cudaStream_t stream);
+                      float *partial, uint32_t *status, bool bf16, cudaStream_t stream);
 
 // Multi-variant prefill: x_sorted holds the token rows in bucket order (contiguous, pitch d_in); token tile
 // i of tile_table is {variant (V = base only), first sorted row, rows (<= token_tile), 0}; token_tile is 64, 128

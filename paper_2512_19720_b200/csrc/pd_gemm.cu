@@ -66,6 +66,10 @@ struct GemmArgs {
     int y_vec_ok;  // y is 16-byte aligned and ldy a multiple of 8: rows can be written with 16-byte stores
     int token_tile;  // pair kernel, one variant: tokens per tile (64, 128 or 256)
     int bf16;        // host side only: which instantiation to launch
+    // pair kernel, one variant: the k steps are dealt to `splits` tiles (k_steps counts one split's steps); with
+    // splits > 1 a tile writes its fp32 partial sums to partial[split][token][row] and splitk_reduce_kernel adds them
+    int splits;
+    float *partial;
 };
 
 struct Tile {
@@ -504,6 +508,7 @@ __device__ __forceinline__ void tcgen05_mma_f16_tmem_a_pair(uint32_t d_tmem, uin
 // Tile of the pair kernel as one CTA sees it.  `half` = token rows each CTA holds in shared memory (MMA N = 2 half).
 struct PairTile {
     int tm, tok0, count, half;   // this CTA's W row tile of 128; first token row; valid tokens; tokens per CTA
+    int k0, split;               // first k step of the tile (split-K), and which split it is
     const uint32_t *mask;
     const __half *v;
     bool col, delta;
@@ -511,6 +516,12 @@ struct PairTile {
 template <int AXIS, bool HAS_DELTA, bool GROUPED>
 __device__ __forceinline__ PairTile get_pair_tile(const GemmArgs &a, int tile, int n_tt, uint32_t rank) {
     PairTile t;
+    t.k0 = 0, t.split = 0;
+    if (!GROUPED && a.splits > 1) {  // the splits of one output tile are neighbours: they share the x tile and finish together
+        t.split = tile % a.splits;
+        tile /= a.splits;
+        t.k0 = t.split * a.k_steps;
+    }
     const int tp = tile / n_tt, tn = tile - tp * n_tt;
     t.tm = 2 * tp + static_cast<int>(rank);
     if (!GROUPED) {  // MMA N = the tile's tokens rounded up to a multiple of 32
@@ -554,7 +565,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int tiles_m2 = (a.tiles_m + 1) >> 1;        // tiles of 256 rows
     const int n_tt = GROUPED ? __ldg(a.n_token_tiles) : a.tiles_n;  // token tiles
-    const int n_tiles = tiles_m2 * n_tt;
+    const int n_tiles = tiles_m2 * n_tt * (GROUPED ? 1 : a.splits);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < L::kStages; ++s) {
@@ -602,15 +613,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                             }
                             if (rank == 0) mbar_arrive_expect_tx(ready + pi % kPairSlots, 4 * L::kXBytes);  // both halves of both steps
                         }
-                        tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes, ks * BK,
-                                         ti.tok0 + ti.half * static_cast<int>(rank));
+                        tma_load_2d_pair(&map_x, map_to_rank(ready + pi % kPairSlots, 0), smem + L::kXOffset + s * L::kXBytes,
+                                         (ti.k0 + ks) * BK, ti.tok0 + ti.half * static_cast<int>(rank));
                     } else {
                         const uint32_t parity = ((it / L::kStages) & 1) ^ 1;
                         if (!(ok = mbar_wait(w_empty + s, parity, abort_flag, a.status, 6))) break;
-                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ks * BK)) * 2) : 0u;
+                        const int ka = ti.k0 + ks;
+                        const uint32_t v_bytes = (ti.delta && ti.col) ? static_cast<uint32_t>(max(0, min(BK, a.d_in - ka * BK)) * 2) : 0u;
                         mbar_arrive_expect_tx(w_full + s, L::kWBytes + v_bytes);
-                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ks * BK, ti.tm * BM);
-                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ks) * BK, v_bytes, w_full + s);
+                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kWBytes, ka * BK, ti.tm * BM);
+                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * kVSlotBytes, ti.v + static_cast<size_t>(ka) * BK, v_bytes, w_full + s);
                     }
                 }
             }
@@ -675,6 +687,30 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const int o0 = ti.tm * BM;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const int n_half = (count + 127) / 128;
+            if (!GROUPED && a.splits > 1) {
+                // split-K: the fp32 partial sums go to partial[split][token][row]; a lane owns a row, so the 32 lanes of
+                // a warp write 128 contiguous bytes per token
+                const int o = o0 + row_l;
+                float *dst = a.partial + (static_cast<size_t>(ti.split) * a.M + tok0) * a.d_out + o;
+                for (int hf = 0; hf < n_half; ++hf) {
+#pragma unroll 1
+                    for (int c0 = kColsPerWarp * col_half; c0 < kColsPerWarp * (col_half + 1); c0 += 32) {
+                        if (hf * 128 + c0 >= count) break;
+                        uint32_t r[32];
+                        tcgen05_ld_32x32b_x32(taddr + hf * 128 + c0, r);
+                        tcgen05_wait_ld();
+                        if (o < a.d_out) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (hf * 128 + c0 + j < count) dst[static_cast<size_t>(hf * 128 + c0 + j) * a.d_out] = __uint_as_float(r[j]);
+                        }
+                    }
+                }
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(acc_empty_rank0);
+                continue;
+            }
             for (int hf = 0; hf < n_half; ++hf) {
 #pragma unroll 1
                 for (int c0 = kColsPerWarp * col_half; c0 < kColsPerWarp * (col_half + 1); c0 += 32) {
@@ -731,9 +767,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 vrow = Elem<BF16>::scale_pair(*reinterpret_cast<const unsigned short *>(ti.v + o));
             }
             const uint32_t *mrow = delta ? ti.mask + static_cast<size_t>(row_ok ? o : 0) * words : nullptr;
+            const int k0 = ti.k0;
             auto load_words = [&](int ks, uint32_t &w0, uint32_t &w1) {
-                w0 = (delta && row_ok && ks < a.k_steps && 2 * ks < words) ? __ldg(mrow + 2 * ks) : 0u;
-                w1 = (delta && row_ok && ks < a.k_steps && 2 * ks + 1 < words) ? __ldg(mrow + 2 * ks + 1) : 0u;
+                w0 = (delta && row_ok && ks < a.k_steps && 2 * (k0 + ks) < words) ? __ldg(mrow + 2 * (k0 + ks)) : 0u;
+                w1 = (delta && row_ok && ks < a.k_steps && 2 * (k0 + ks) + 1 < words) ? __ldg(mrow + 2 * (k0 + ks) + 1) : 0u;
             };
             int ks = static_cast<int>((par ^ it) & 1u);
             uint32_t q0[4], q1[4];
@@ -786,6 +823,38 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     }
 }
 
+
+// Split-K: y[token][row] = sum over the splits, in split order, of partial[split][token][row], rounded once to the
+// storage type.  Four rows per thread.
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *partial, int splits, int M, int d_out, __half *y, int64_t ldy, int vec_ok) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // launched while the GEMM still runs
+    const int per_row = (d_out + 3) >> 2;
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+    if (idx >= static_cast<int64_t>(M) * per_row) return;
+    const int tok = static_cast<int>(idx / per_row), o = static_cast<int>(idx - static_cast<int64_t>(tok) * per_row) * 4;
+    const size_t plane = static_cast<size_t>(M) * d_out;
+    const float *src = partial + static_cast<size_t>(tok) * d_out + o;
+    unsigned short *dst = reinterpret_cast<unsigned short *>(y) + static_cast<size_t>(tok) * ldy + o;
+    if (vec_ok) {
+        float4 acc = *reinterpret_cast<const float4 *>(src);
+        for (int sp = 1; sp < splits; ++sp) {
+            const float4 t = *reinterpret_cast<const float4 *>(src + sp * plane);
+            acc.x += t.x, acc.y += t.y, acc.z += t.z, acc.w += t.w;
+        }
+        uint2 out;
+        out.x = Elem<BF16>::from_float(acc.x) | (static_cast<uint32_t>(Elem<BF16>::from_float(acc.y)) << 16);
+        out.y = Elem<BF16>::from_float(acc.z) | (static_cast<uint32_t>(Elem<BF16>::from_float(acc.w)) << 16);
+        *reinterpret_cast<uint2 *>(dst) = out;
+    } else {
+        for (int q = 0; q < 4 && o + q < d_out; ++q) {
+            float acc = src[q];
+            for (int sp = 1; sp < splits; ++sp) acc += src[sp * plane + q];
+            dst[q] = Elem<BF16>::from_float(acc);
+        }
+    }
+}
 
 // ------------------------------------------------------------------ host side
 }  // namespace
@@ -881,8 +950,8 @@ pd_status launch_pair_one(const CUtensorMap &mw, const CUtensorMap &mx, const Ge
 
 // Tiles of 256 rows x 256 tokens on pairs of CTAs.
 pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask, const __half *v,
-                           int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, int token_tile, uint32_t *status,
-                           bool bf16, cudaStream_t stream) {
+                           int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy, int token_tile, int splits,
+                           float *partial, uint32_t *status, bool bf16, cudaStream_t stream) {
     CUtensorMap mw, mx;
     if (!make_map(&mw, w_b, d_out, d_in, d_in, BM) || !make_map(&mx, x, M, d_in, ldx, 128)) return PD_ERR_CUDA;
     GemmArgs args = {};
@@ -896,15 +965,35 @@ pd_status launch_gemm_pair(const __half *x, int64_t M, int64_t ldx, const __half
     args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
     args.tiles_n = static_cast<int>((M + token_tile - 1) / token_tile);
     args.token_tile = token_tile;
-    args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;  // even: the MMA thread works on pairs of k steps
+    args.k_steps = pair_split_steps(d_in, splits);  // per split; even: the MMA thread works on pairs of k steps
+    args.splits = splits;
+    args.partial = partial;
     args.status = status;
     args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
-    const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n;
+    const int tiles = ((args.tiles_m + 1) / 2) * args.tiles_n * splits;
     const int pairs = tiles < sm_count() / 2 ? tiles : sm_count() / 2;
-    if (mask == nullptr) return launch_pair_one<PD_AXIS_ROW, false, false>(mw, mx, args, 2 * pairs, stream);
-    if (axis == PD_AXIS_ROW) return launch_pair_one<PD_AXIS_ROW, true, false>(mw, mx, args, 2 * pairs, stream);
-    return launch_pair_one<PD_AXIS_COL, true, false>(mw, mx, args, 2 * pairs, stream);
+    pd_status st;
+    if (mask == nullptr) st = launch_pair_one<PD_AXIS_ROW, false, false>(mw, mx, args, 2 * pairs, stream);
+    else if (axis == PD_AXIS_ROW) st = launch_pair_one<PD_AXIS_ROW, true, false>(mw, mx, args, 2 * pairs, stream);
+    else st = launch_pair_one<PD_AXIS_COL, true, false>(mw, mx, args, 2 * pairs, stream);
+    if (st != PD_OK || splits == 1) return st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // scheduled while the GEMM runs; it waits on entry
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    const int64_t threads = M * ((d_out + 3) / 4);
+    cfg.gridDim = dim3(static_cast<unsigned>((threads + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int vec_ok = (d_out % 4 == 0 && ldy % 4 == 0 && (reinterpret_cast<uintptr_t>(y) & 7u) == 0) ? 1 : 0;
+    const int m32 = static_cast<int>(M), d32 = static_cast<int>(d_out);
+    const float *cpartial = partial;
+    count_launch();
+    return cuda_ok(bf16 ? cudaLaunchKernelEx(&cfg, splitk_reduce_kernel<true>, cpartial, splits, m32, d32, y, ldy, vec_ok)
+                        : cudaLaunchKernelEx(&cfg, splitk_reduce_kernel<false>, cpartial, splits, m32, d32, y, ldy, vec_ok));
 }
 
 // Multi-variant: token tiles of at most 256 sorted rows, one variant each.
@@ -926,6 +1015,7 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
     args.tiles_m = static_cast<int>((d_out + BM - 1) / BM);
     args.tiles_n = 0;
     args.k_steps = static_cast<int>((d_in + 2 * BK - 1) / (2 * BK)) * 2;
+    args.splits = 1;
     args.status = status;
     args.bf16 = bf16 ? 1 : 0;
     args.y_vec_ok = ((reinterpret_cast<uintptr_t>(y) & 15u) == 0 && ldy % 8 == 0) ? 1 : 0;
@@ -943,25 +1033,57 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
 
 }  // namespace
 
+namespace {
+
+// Token tile and number of k splits of the pair kernel.  A pair of k steps costs the issuing thread about 1250 clocks
+// whatever the tile's width (the MMA instruction rate) and the tensor cores 4 clocks per token; a tile costs about
+// 3000 clocks to start and drain.  With few tokens the tiles are too few for the 74 CTA pairs: the k steps are then
+// dealt to several tiles whose fp32 partial sums a second kernel adds (about 5000 clocks plus its traffic).  Picks
+// the cheapest estimate; ties go to fewer splits, then to the narrower tile (more CTAs stream the weights).
+void pair_plan(int64_t M, int64_t d_out, int64_t d_in, int sms, int *token_tile, int *splits) {
+    const int64_t tiles_m2 = (d_out + 2 * BM - 1) / (2 * BM);
+    const int pairs = sms / 2 > 0 ? sms / 2 : 1;
+    const int64_t k_pairs = (d_in + 2 * BK - 1) / (2 * BK);
+    int64_t best_cost = -1;
+    for (int sp = 1; sp <= 8; ++sp) {
+        if (sp > 1 && (M > 1024 || k_pairs / sp < 4)) break;
+        for (int tt = 256; tt >= 64; tt >>= 1) {
+            const int64_t units = tiles_m2 * ((M + tt - 1) / tt) * sp;
+            const int64_t per_pair = 4 * tt + 400 > 1250 ? 4 * tt + 400 : 1250;
+            const int64_t per_unit = ((k_pairs + sp - 1) / sp) * per_pair + 3000;
+            int64_t cost = ((units + pairs - 1) / pairs) * per_unit;
+            if (sp > 1) cost += 5000 + (M * d_out * (sp + 1)) / 2048;  // the reduction: ~4 bytes per partial at ~2 KB per clock
+            if (best_cost < 0 || cost < best_cost || (cost == best_cost && sp == *splits)) *token_tile = tt, *splits = sp, best_cost = cost;
+        }
+    }
+}
+
+}  // namespace
+
+int pair_split_steps(int64_t d_in, int splits) {
+    const int64_t k_pairs = (d_in + 2 * BK - 1) / (2 * BK);
+    return static_cast<int>((k_pairs + splits - 1) / splits) * 2;
+}
+
+size_t gemm_partial_bytes(int64_t M, int64_t d_out, int64_t d_in) {
+    if (!(gemm_pair_enabled() && d_out >= 256)) return 0;
+    int tt = 256, splits = 1;
+    pair_plan(M, d_out, d_in, sm_count(), &tt, &splits);
+    return splits > 1 ? round_up(static_cast<size_t>(splits) * M * d_out * 4, 256) : 0;
+}
+
 pd_status launch_gemm(const __half *x, int64_t M, int64_t ldx, const __half *w_b, const uint32_t *mask,
                       const __half *v, int axis, int64_t d_out, int64_t d_in, __half *y, int64_t ldy,
-                      uint32_t *status, bool bf16, cudaStream_t stream) {
+                      float *partial, uint32_t *status, bool bf16, cudaStream_t stream) {
     const int sms = sm_count();
     if (gemm_pair_enabled() && d_out >= 256) {
         // CTA pairs, tiles of 256 rows x token_tile tokens.  A pair of k steps costs the issuing thread about 1250
         // clocks whatever the tile's width (the MMA instruction rate), the tensor cores 4 clocks per token; pick the
         // width with the fewest rounds x that, ties to the narrower tile (more CTAs stream the weights).
-        const int64_t tiles_m2 = (d_out + 2 * BM - 1) / (2 * BM);
-        const int pairs = sms / 2;
-        int best_tt = 256;
-        int64_t best_tt_cost = -1;
-        for (int tt = 256; tt >= 64; tt >>= 1) {
-            const int64_t units = tiles_m2 * ((M + tt - 1) / tt);
-            const int64_t per = 4 * tt + 400 > 1250 ? 4 * tt + 400 : 1250;
-            const int64_t cost = ((units + pairs - 1) / pairs) * per;
-            if (best_tt_cost < 0 || cost <= best_tt_cost) best_tt = tt, best_tt_cost = cost;
-        }
-        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, best_tt, status, bf16, stream);
+        int tt = 256, splits = 1;
+        pair_plan(M, d_out, d_in, sms, &tt, &splits);
+        if (splits > 1 && partial == nullptr) return PD_ERR_WORKSPACE;
+        return launch_gemm_pair(x, M, ldx, w_b, mask, v, axis, d_out, d_in, y, ldy, tt, splits, partial, status, bf16, stream);
     }
     // One CTA per tile (fewer than 256 output rows).  256 tokens per tile amortise the W_hat transform best, but with
     // few tokens that leaves most SMs without
