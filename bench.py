@@ -53,10 +53,12 @@ MULTI_M = (64, 64 + 4 * 512)
 FIT_M = 2048  # calibration tokens per training step of the scale fit
 C1_COPIES = 128
 ROW, COL = 0, 1
-# ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the captures summarised in profiles/;
-# None = the kernel has changed since its counters were taken (merge: reads only -- half of its writes are still
-# dirty in L2 when the kernel ends)
-NCU_DRAM_RATIO = {"decode": None, "pack": None, "merge": 1.0, "multi_decode": None}
+# ncu dram bytes / algorithmic bytes of the captures summarised in profiles/ (4096x11008 for the streaming kernels,
+# 4096x4096 with 64 tokens over 16 variants for the multi-variant decode; their traffic grows in proportion to the
+# elements streamed).  Pack and multi-variant decode: read + write.  Decode GEMV and merge: the read ratio -- the GEMV
+# writes 8 KB, what ncu counts as its writes is earlier data leaving the L2, and half of merge's writes are still dirty
+# in L2 when the kernel ends.  None = the kernel has changed since its counters were taken.
+NCU_DRAM_RATIO = {"decode": 1.004, "pack": 0.996, "merge": 1.0, "multi_decode": 0.987}
 METRIC = "fused delta-linear decode HBM GB/s (7B block sweep, M in {1,4,16}, row+col axes)"
 
 
@@ -447,8 +449,8 @@ def run_ours(args):
         "gemv_stream_kernel<bf16>")
     add("bf16_prefill_m2048", lambda: bf_linear((2048,), False), 2 * flops(2048), "TFLOP/s", 14, "gemm_pair_kernel<bf16>")
     add("bf16_merge", bf_merge, S["merge"]["work"], "GB/s", 14, "merge_kernel<bf16>")
-    add("fit_row_m2048", lambda: run_fit(ROW), 2 * 2 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<row> (two tcgen05 accumulators)")
-    add("fit_col_m2048", lambda: run_fit(COL), 3 * 2 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<col forward>, <col backward>")
+    add("fit_row_m2048", lambda: run_fit(ROW), 2 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<row> (two tcgen05 accumulators)")
+    add("fit_col_m2048", lambda: run_fit(COL), 3 * flops(FIT_M), "TFLOP/s", 7, "fit_gemm_kernel<col forward>, <col backward>")
     for m in (1, 16):
         for rotated in (True, False):
             add(f"c1_m{m}_{'rotated' if rotated else 'resident'}", lambda m=m, r=rotated: run_c1(m, r),
@@ -726,11 +728,19 @@ def run_only(args):
     x = synth_torch.gen_x(args.m, d_in, 5, dev)
     y = torch.empty((args.m, d_out), dtype=torch.float16, device=dev)
     ids = synth_torch.gen_ids(args.m, N_VARIANTS, 3000 + args.m, dev)
+    if args.only == "fit":
+        y_fit = [(x @ L[1].T).contiguous() for L in layers]
+        mask_t = [api.pd_transpose_mask(L[2], d_out, d_in) for L in layers]
+        v32 = [L[3][axis].float().contiguous() for L in layers]
+        fit_loss, fit_grad = torch.zeros(1, device=dev), torch.zeros_like(v32[0])
 
     def call(i):
         L = layers[i % copies]
         w_b, w_f, mask, v, out = L[:5]
-        if args.only == "linear":
+        if args.only == "fit":
+            c = i % copies
+            api.pd_fit_loss_grad(x, y_fit[c], w_b, mask, v32[c], axis, mask_t=mask_t[c], loss=fit_loss, grad=fit_grad)
+        elif args.only == "linear":
             api.pd_linear(x, w_b, mask, v[axis], axis, y=y, weights_resident=True)
         elif args.only == "pack":
             api.pd_pack_delta(w_f, w_b, mask=mask, v_row=v[0], v_col=v[1])
@@ -761,7 +771,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-config5", action="store_true", help="leave the 70B-shaped sections out (they need ~6 GB and ~0.2 s per step)")
-    ap.add_argument("--only", choices=["linear", "pack", "merge", "multi"], help="run one kernel family on one layer (for profiling)")
+    ap.add_argument("--only", choices=["linear", "pack", "merge", "multi", "fit"], help="run one kernel family on one layer (for profiling)")
     ap.add_argument("--shape", default="4096x4096")
     ap.add_argument("--m", type=int, default=16)
     ap.add_argument("--axis", default="row", choices=["row", "col"])

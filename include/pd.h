@@ -106,7 +106,9 @@ pd_status pd_pack_delta(const void *w_f, const void *w_b, int64_t d_out, int64_t
  * products are accumulated in fp32 and y is rounded to fp16 once at the end.  M <= 16 runs the
  * bandwidth-bound decode kernel, larger M the tensor-core (tcgen05) kernel, which needs d_out and
  * d_in to be multiples of 8 and d_in >= 64 (otherwise the rows go through the decode kernel in
- * chunks of 16).  Needs pd_workspace_bytes(PD_OP_LINEAR, M, ...).
+ * chunks of 16).  Needs pd_workspace_bytes(PD_OP_LINEAR, M, 0, d_out, d_in) bytes: the status words and, when M is
+ * small against the number of SMs (up to about a thousand tokens), fp32 partial sums of a k loop that is dealt to
+ * several thread blocks and added in a fixed order by a second kernel (the result does not depend on the schedule).
  */
 pd_status pd_linear(const void *x, int64_t M, int64_t ldx,
                     const void *w_b, const uint32_t *mask, const void *v, pd_axis axis,
