@@ -299,7 +299,7 @@ pd_status pd_selftest_bounded_wait(void *workspace, int64_t limit_cycles, void *
  * n = M * d_out (the mean over all output entries).  W_b, x, y are fp16; v, gradients and optimiser state are fp32
  * device arrays; every product runs on the tensor cores with fp32 accumulation, W_b and the sign matrix as separate
  * operands.  Sizes: d_in a multiple of 32, d_out a multiple of 8, M >= 1; x [M, d_in] and y [M, d_out] contiguous,
- * x and w_b 16-byte aligned.  All calls enqueue on the stream and return; errors the device latches (a bounded wait
+ * x, y and w_b 16-byte aligned.  All calls enqueue on the stream and return; errors the device latches (a bounded wait
  * that ran out) are read with pd_device_status(workspace).
  */
 

@@ -467,7 +467,7 @@ pd_status pd_fit_loss_grad(const void *x, const void *y, int64_t M, const void *
     if (axis == PD_AXIS_COL && grad && !mask_t) return PD_ERR_INVALID_ARG;
     const pd_status shape = fit_shape_check(M, d_out, d_in);
     if (shape != PD_OK) return shape;
-    if (!aligned16(x) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
     if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_FIT, M, 0, d_out, d_in)) return PD_ERR_WORKSPACE;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     return launch_fit_loss_grad(static_cast<const __half *>(x), static_cast<const __half *>(y), M, static_cast<const __half *>(w_b), mask,
@@ -493,7 +493,8 @@ pd_status pd_fit_layer(const void *x_tr, const void *y_tr, int64_t M_tr, const v
     if (shape == PD_OK) shape = fit_shape_check(M_val, d_out, d_in);
     if (shape != PD_OK) return shape;
     if ((d_out + 31) / 32 > 65535) return PD_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned16(x_tr) || !aligned16(x_val) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
+    if (!aligned16(x_tr) || !aligned16(x_val) || !aligned16(y_tr) || !aligned16(y_val) || !aligned16(w_b)) return PD_ERR_ALIGNMENT;
+    if ((batch * d_out) % 8 != 0 && batch < M_tr) return PD_ERR_ALIGNMENT;  // every minibatch of y starts 16-byte aligned
     if (batch > M_tr) batch = M_tr;
     const int64_t m_max = batch > M_val ? batch : M_val;
     if (!workspace || !aligned256(workspace) || workspace_bytes < pd_workspace_bytes(PD_OP_FIT_LAYER, m_max, 0, d_out, d_in))

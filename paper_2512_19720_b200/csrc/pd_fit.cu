@@ -9,33 +9,38 @@
 // Every product runs on the 5th-generation tensor cores with fp32 accumulation; W_b and B are separate operands
 // (B as exact +-1, or +-binary16(v[i]) for the col axis), so the delta term is not rounded into the weights.
 // One kernel, three modes:
-//   FIT_ROW_FWD : two accumulators (Z, P) per tile of 128 rows x 128 tokens; the epilogue forms R, the squared
+//   FIT_ROW_FWD : two accumulators (Z, P) per tile of 128 rows x 192 tokens; the epilogue forms R, the squared
 //                 error and the row gradient without writing R anywhere
 //   FIT_COL_FWD : one accumulator; the epilogue writes R as binary16 for the second pass
 //   FIT_COL_BWD : T^T = B^T R^T from the transposed mask (rows = input columns); the epilogue multiplies by X
-// Roles, rings and barriers follow the prefill kernel: warp 0 TMA of the token operand, warp 1 MMA issue, warps 2-5
-// epilogue, warps 6-13 expand the weight-side operands into tensor memory (a thread owns one row = one TMEM lane),
-// warp 14 TMA of the W_b tile.  A k step is 64 wide; its two operand slots (W_b rows, sign rows) are 64 TMEM
-// columns; four k steps are in flight.  Partial sums go to the workspace per tile and are added in a fixed order by
-// fit_reduce_kernel: results do not depend on the schedule.  Every wait is bounded.
+// A tcgen05.mma costs its issuing thread about 150 clocks whatever its N, so the tiles are as wide in tokens as tensor
+// memory allows in the row mode: 2 x 192 accumulator columns + the sign ring (4 x 32).  The tile of Y (of X in the
+// backward mode) that the epilogue needs is fetched into shared memory with cp.async while the tile's MMAs run:
+// read element by element from global memory it cost 40 % of the kernel's time.
+// The W_b tile is an MMA operand straight from the shared memory TMA filled (A from a shared-memory descriptor);
+// only the sign rows go through tensor memory: a thread of the eight transform warps owns one row (= one TMEM lane)
+// and expands two mask words per 64-wide k step.  Roles: warp 0 TMA (token tile, W_b tile, the col-axis scales of
+// the step), warp 1 MMA issue, warps 2-5 epilogue, warps 6-13 transform.  Four k steps are in flight.  Partial sums
+// go to the workspace per tile and are added in a fixed order by fit_reduce_kernel: results do not depend on the
+// schedule.  Every wait is bounded.
 #include "pd_tcgen05.cuh"
 
 namespace pd {
 namespace {
 
 constexpr int FM = 128;           // rows of the weight-side operand per tile (MMA M, TMEM lanes)
-constexpr int FN = 128;           // tokens per tile (MMA N)
 constexpr int FK = 64;            // k per step
-constexpr int kFitStages = 4;     // token ring, W_b ring and operand ring (tensor memory)
-constexpr int kFitWarps = 15;
+constexpr int kFitStages = 4;     // token ring, W_b ring and sign ring (tensor memory)
+constexpr int kFitWarps = 14;
 constexpr int kFitThreads = kFitWarps * 32;
 constexpr int kFitXformWarps = 8;
 constexpr int kFitEpiWarps = 4;
-constexpr int kFitAccP = FN;          // TMEM column of the second accumulator
-constexpr int kFitACol0 = 2 * FN;     // operand ring: kFitStages slots of 64 columns
+constexpr int kFitACol0 = 384;        // sign ring: kFitStages slots of 32 TMEM columns
 constexpr uint32_t kOnesF16 = 0x3C003C00u;
 
 enum FitMode { FIT_ROW_FWD = 0, FIT_COL_FWD = 1, FIT_COL_BWD = 2 };
+// tokens per tile (MMA N): the row mode keeps two accumulators in 384 of the 512 tensor-memory columns
+__host__ __device__ constexpr int fit_tokens(int) { return 192; }
 
 struct FitArgs {
     const uint32_t *bits;  // forward: mask [d_out][d_in/32]; backward: transposed mask [d_in][words_t]
@@ -55,14 +60,30 @@ struct FitArgs {
 };
 
 struct FitSmem {
-    static constexpr int kTileBytes = FM * FK * 2;  // 16 KB: token tile and W_b tile alike
+    static constexpr int kXBytes = fit_tokens(0) * FK * 2;   // 24 KB
+    static constexpr int kWBytes = FM * FK * 2;              // 16 KB
     static constexpr int kXOffset = 0;
-    static constexpr int kWOffset = kFitStages * kTileBytes;
-    static constexpr int kBarOffset = 2 * kFitStages * kTileBytes;
+    static constexpr int kWOffset = kFitStages * kXBytes;
+    static constexpr int kYOffset = kWOffset + kFitStages * kWBytes;   // [token][128 rows] binary16: the epilogue's Y (or X) tile
+    static constexpr int kYBytes = fit_tokens(0) * FM * 2;   // 48 KB
+    static constexpr int kBarOffset = kYOffset + kYBytes;
     static constexpr int kVOffset = kBarOffset + 256;          // col forward: the 64 scales of a k step, per stage
     static constexpr int kRedOffset = kVOffset + kFitStages * 128;
     static constexpr int kTotal = kRedOffset + 64 + 1024;      // + slack for 1024-byte alignment
+    static_assert(kTotal <= 227 * 1024, "shared memory per CTA");
 };
+
+// A from shared memory (K-major tile, 128-byte swizzle, like B)
+__device__ __forceinline__ void tcgen05_mma_f16_smem_a(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                       uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 
 // 64 signs (two mask words) -> 32 registers of two binary16 each: +mag where the bit is 1, -mag where it is 0.
 // COL: mag = the step's 64 scales from shared memory; else mag = 1.
@@ -86,13 +107,17 @@ template <int MODE>
 __global__ void __launch_bounds__(kFitThreads, 1)
 fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const FitArgs a) {
     constexpr bool FWD = MODE != FIT_COL_BWD;
+    constexpr int BN = fit_tokens(MODE);
+    constexpr uint32_t kAccP = BN;  // TMEM column of the second accumulator (row mode)
+    static_assert((MODE == FIT_ROW_FWD ? 2 : 1) * BN <= kFitACol0, "accumulators end where the sign ring starts");
     using L = FitSmem;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::kBarOffset);
-    uint64_t *w_full = bars, *w_empty = bars + kFitStages;
-    uint64_t *ready = bars + 2 * kFitStages, *consumed = bars + 3 * kFitStages;
-    uint64_t *acc_full = bars + 4 * kFitStages, *acc_empty = acc_full + 1;
+    uint64_t *v_full = bars;                       // col forward: the step's scales have landed
+    uint64_t *ready = bars + kFitStages;           // token tile and W_b tile landed (TMA bytes + the producer's arrival), sign slot written
+    uint64_t *consumed = bars + 2 * kFitStages;    // the MMAs of the step have read its shared-memory tiles and its sign slot
+    uint64_t *acc_full = bars + 3 * kFitStages, *acc_empty = acc_full + 1;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     float *red = reinterpret_cast<float *>(smem + L::kRedOffset);
@@ -102,8 +127,7 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kFitStages; ++s) {
-            mbar_init(w_full + s, 1);
-            mbar_init(w_empty + s, kFitXformWarps / 2);
+            mbar_init(v_full + s, 1);
             mbar_init(ready + s, kFitXformWarps / 2 + 1);
             mbar_init(consumed + s, 1);
         }
@@ -122,10 +146,9 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0 || warp == kFitWarps - 1) {
-        // ------------------------------------------------ TMA producers: warp 0 the token operand, the last warp W_b
-        const bool is_x = warp == 0;
-        if (lane == 0 && (is_x || FWD)) {
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer: token tile, W_b tile, col-axis scales of the step
+        if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -133,24 +156,23 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                 for (int ks = 0; ks < a.k_steps; ++ks, ++it) {
                     const int s = it % kFitStages;
                     const uint32_t round = it / kFitStages;
-                    if (is_x) {
-                        if (round > 0 && !(ok = mbar_wait(consumed + s, (round - 1) & 1, abort_flag, a.status, 31))) break;
-                        mbar_arrive_expect_tx(ready + s, L::kTileBytes);
-                        tma_load_2d(&map_x, ready + s, smem + L::kXOffset + s * L::kTileBytes, ks * FK, tn * FN);
-                    } else {
-                        if (!(ok = mbar_wait(w_empty + s, (round & 1) ^ 1, abort_flag, a.status, 32))) break;
-                        const uint32_t v_bytes = MODE == FIT_COL_FWD ? static_cast<uint32_t>(min(FK, a.K - ks * FK) * 2) : 0u;
-                        mbar_arrive_expect_tx(w_full + s, L::kTileBytes + v_bytes);
-                        tma_load_2d(&map_w, w_full + s, smem + L::kWOffset + s * L::kTileBytes, ks * FK, tm * FM);
-                        if (v_bytes) bulk_load_1d(smem + L::kVOffset + s * 128, a.v16 + static_cast<size_t>(ks) * FK, v_bytes, w_full + s);
+                    // the slots were last read by k step it - kFitStages
+                    if (round > 0 && !(ok = mbar_wait(consumed + s, (round - 1) & 1, abort_flag, a.status, 31))) break;
+                    if (MODE == FIT_COL_FWD) {
+                        const uint32_t v_bytes = static_cast<uint32_t>(min(FK, a.K - ks * FK) * 2);
+                        mbar_arrive_expect_tx(v_full + s, v_bytes);
+                        bulk_load_1d(smem + L::kVOffset + s * 128, a.v16 + static_cast<size_t>(ks) * FK, v_bytes, v_full + s);
                     }
+                    mbar_arrive_expect_tx(ready + s, BN * FK * 2 + (FWD ? L::kWBytes : 0));
+                    tma_load_2d(&map_x, ready + s, smem + L::kXOffset + s * L::kXBytes, ks * FK, tn * BN);
+                    if (FWD) tma_load_2d(&map_w, ready + s, smem + L::kWOffset + s * L::kWBytes, ks * FK, tm * FM);
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = kIdescBase<false> | (static_cast<uint32_t>(FN >> 3) << 17) | (static_cast<uint32_t>(FM >> 4) << 24);
+            const uint32_t idesc = kIdescBase<false> | (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(FM >> 4) << 24);
             uint32_t it = 0, tcount = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
@@ -160,17 +182,18 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                     const int s = it % kFitStages;
                     if (!(ok = mbar_wait(ready + s, (it / kFitStages) & 1, abort_flag, a.status, 34))) break;
                     tcgen05_fence_after();
-                    const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kTileBytes);
-                    const uint32_t a_w = tmem_base + kFitACol0 + s * 64, a_s = a_w + 32;
+                    const uint32_t x_addr = smem_u32(smem + L::kXOffset + s * L::kXBytes);
+                    const uint32_t w_addr = smem_u32(smem + L::kWOffset + s * L::kWBytes);
+                    const uint32_t a_s = tmem_base + kFitACol0 + s * 32;
 #pragma unroll
                     for (int kk = 0; kk < FK / 16; ++kk) {
                         const uint64_t xd = make_smem_desc(x_addr + kk * 32);
                         const uint32_t first = (ks > 0 || kk > 0) ? 1u : 0u;
                         if (MODE == FIT_ROW_FWD) {
-                            tcgen05_mma_f16_tmem_a(tmem_base, a_w + kk * 8, xd, idesc, first);
-                            tcgen05_mma_f16_tmem_a(tmem_base + kFitAccP, a_s + kk * 8, xd, idesc, first);
+                            tcgen05_mma_f16_smem_a(tmem_base, make_smem_desc(w_addr + kk * 32), xd, idesc, first);
+                            tcgen05_mma_f16_tmem_a(tmem_base + kAccP, a_s + kk * 8, xd, idesc, first);
                         } else if (MODE == FIT_COL_FWD) {
-                            tcgen05_mma_f16_tmem_a(tmem_base, a_w + kk * 8, xd, idesc, first);
+                            tcgen05_mma_f16_smem_a(tmem_base, make_smem_desc(w_addr + kk * 32), xd, idesc, first);
                             tcgen05_mma_f16_tmem_a(tmem_base, a_s + kk * 8, xd, idesc, 1u);
                         } else {
                             tcgen05_mma_f16_tmem_a(tmem_base, a_s + kk * 8, xd, idesc, first);
@@ -184,9 +207,24 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     } else if (warp < 2 + kFitEpiWarps) {
         // ------------------------------------------------ epilogue: a thread owns one row of the tile and walks its tokens
         const int quarter = warp & 3;
+        const int et = threadIdx.x - 2 * 32;  // 0..127 among the epilogue threads
+        const unsigned char *ybuf = smem + L::kYOffset;
+        const __half *side = FWD ? a.y : a.x;  // [M][rows]: the operand the epilogue combines with the accumulator
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
             const int tm = tile / a.tiles_n, tn = tile - tm * a.tiles_n;
+            {   // this tile's [tokens][128 rows] piece of `side`, 16 bytes per copy, while the MMAs run
+                const int n_tok = min(BN, a.M - tn * BN);
+                for (int idx = et; idx < n_tok * 16; idx += kFitEpiWarps * 32) {
+                    const int tok = idx >> 4, ch = idx & 15;
+                    const int r8 = tm * FM + ch * 8;
+                    if (r8 < a.rows)  // rows is a multiple of 8: a piece is valid as a whole or not at all
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(ybuf + tok * (FM * 2) + ch * 16)),
+                                     "l"(side + static_cast<size_t>(tn * BN + tok) * a.rows + r8)
+                                     : "memory");
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            }
             const bool got = mbar_wait(acc_full, tcount & 1, abort_flag, a.status, 35);
             uint32_t gave_up;  // OR over the epilogue warps, so that they leave together
             asm volatile(
@@ -199,30 +237,33 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                 : "=r"(gave_up)
                 : "r"(static_cast<uint32_t>(!got)), "n"(kFitEpiWarps * 32)
                 : "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
             if (gave_up) break;
+            asm volatile("bar.sync 2, %0;" ::"n"(kFitEpiWarps * 32) : "memory");  // every thread's copies have landed
             tcgen05_fence_after();
             const int row = tm * FM + quarter * 32 + lane;
             const bool row_ok = row < a.rows;
-            const int tok0 = tn * FN;
-            const int count = min(FN, a.M - tok0);
+            const __half *ycol = reinterpret_cast<const __half *>(ybuf) + quarter * 32 + lane;  // + token * FM
+            const int tok0 = tn * BN;
+            const int count = min(BN, a.M - tok0);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             float vo = 0.f;
             if (MODE == FIT_ROW_FWD && row_ok) vo = __ldg(a.v + (a.scalar ? 0 : row));
             float g_acc = 0.f, l_acc = 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < FN; c0 += 32) {
+            for (int c0 = 0; c0 < BN; c0 += 32) {
                 if (c0 >= count) break;  // warp-uniform
                 uint32_t z[32];
                 tcgen05_ld_32x32b_x32(taddr + c0, z);
                 if (MODE == FIT_ROW_FWD) {
                     uint32_t p[32];
-                    tcgen05_ld_32x32b_x32(taddr + kFitAccP + c0, p);
+                    tcgen05_ld_32x32b_x32(taddr + kAccP + c0, p);
                     tcgen05_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int tok = tok0 + c0 + j;
                         if (row_ok && tok < a.M) {
-                            const float yv = __half2float(__ldg(a.y + static_cast<size_t>(tok) * a.rows + row));
+                            const float yv = __half2float(ycol[(c0 + j) * FM]);
                             const float pj = __uint_as_float(p[j]);
                             const float r = fmaf(vo, pj, __uint_as_float(z[j])) - yv;
                             l_acc = fmaf(r, r, l_acc);
@@ -235,7 +276,7 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                     for (int j = 0; j < 32; ++j) {
                         const int tok = tok0 + c0 + j;
                         if (row_ok && tok < a.M) {
-                            const float yv = __half2float(__ldg(a.y + static_cast<size_t>(tok) * a.rows + row));
+                            const float yv = __half2float(ycol[(c0 + j) * FM]);
                             const float r = __uint_as_float(z[j]) - yv;
                             l_acc = fmaf(r, r, l_acc);
                             a.resid[static_cast<size_t>(tok) * a.ld_r + row] = __float2half_rn(r);
@@ -247,7 +288,7 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                     for (int j = 0; j < 32; ++j) {
                         const int tok = tok0 + c0 + j;
                         if (row_ok && tok < a.M) {
-                            const float xv = __half2float(__ldg(a.x + static_cast<size_t>(tok) * a.rows + row));
+                            const float xv = __half2float(ycol[(c0 + j) * FM]);
                             g_acc = fmaf(xv, __uint_as_float(z[j]), g_acc);
                         }
                     }
@@ -257,6 +298,7 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty);
             if (MODE != FIT_COL_FWD && row_ok) a.part_g[static_cast<size_t>(tn) * a.rows + row] = g_acc;
+            if (!FWD) asm volatile("bar.sync 2, %0;" ::"n"(kFitEpiWarps * 32) : "memory");  // the tile in shared memory is free again
             if (FWD) {  // squared error of the tile: lanes in a fixed tree, then the four warps in order
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) l_acc += __shfl_xor_sync(0xffffffffu, l_acc, d);
@@ -267,9 +309,9 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
             }
         }
     } else {
-        // ------------------------------------------------ transform: W_b rows pass through, sign rows are expanded
+        // ------------------------------------------------ transform: the sign rows of a k step -> its slot in tensor memory
         const int quarter = warp & 3;
-        const uint32_t par = static_cast<uint32_t>((warp - (2 + kFitEpiWarps)) >> 2);
+        const uint32_t par = static_cast<uint32_t>((warp - (2 + kFitEpiWarps)) >> 2);  // four warps take the even steps, four the odd ones
         const int r = quarter * 32 + lane;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + kFitACol0;
         uint32_t it = 0;
@@ -296,25 +338,16 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                 for (int d = 0; d < 3; ++d) q0[d] = q0[d + 1], q1[d] = q1[d + 1];
                 load_words(ks + 8, q0[3], q1[3]);
                 uint32_t out[32];
-                if (FWD) {
-                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(w_full + s, round & 1, abort_flag, a.status, 36)))) break;
-                    const unsigned char *wt = smem + L::kWOffset + s * L::kTileBytes + r * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint4 w = *reinterpret_cast<const uint4 *>(wt + ((c ^ (r & 7)) << 4));
-                        out[4 * c] = w.x, out[4 * c + 1] = w.y, out[4 * c + 2] = w.z, out[4 * c + 3] = w.w;
-                    }
+                if (MODE == FIT_COL_FWD) {
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(v_full + s, round & 1, abort_flag, a.status, 36)))) break;
+                    build_sign_row<true>(out, smem + L::kVOffset + s * 128, word0, word1);
+                } else {
+                    build_sign_row<false>(out, nullptr, word0, word1);
                 }
+                // the slot was last read by the MMAs of k step my_it - kFitStages
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait(consumed + s, (round & 1) ^ 1, abort_flag, a.status, 37)))) break;
                 tcgen05_fence_after();
-                if (FWD) tcgen05_st_32x32b_x32(a_taddr + s * 64, out);
-                if (MODE == FIT_COL_FWD) build_sign_row<true>(out, smem + L::kVOffset + s * 128, word0, word1);
-                else build_sign_row<false>(out, nullptr, word0, word1);
-                tcgen05_st_32x32b_x32(a_taddr + s * 64 + 32, out);
-                if (FWD) {  // every shared-memory read of the stage has returned: its registers went into the stores
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(w_empty + s);
-                }
+                tcgen05_st_32x32b_x32(a_taddr + s * 32, out);
                 tcgen05_wait_st();
                 tcgen05_fence_before();
                 __syncwarp();
@@ -337,7 +370,6 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
         tcgen05_dealloc(tmem_base, 512);
     }
 }
-
 
 // Adds the per-tile partial sums in a fixed order (double accumulation) and applies the factors of the mean:
 // grad[k] = (2/n) sum over token tiles of part_g[tile][k]; the block after the gradient blocks writes
@@ -437,8 +469,8 @@ fit_select_kernel(const float *val_loss, const float *v_row, int d_out, const fl
     if (blockIdx.x == 0 && threadIdx.x == 0) *axis_out = row ? PD_AXIS_ROW : PD_AXIS_COL;
 }
 
-bool make_fit_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld) {
-    return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, rows, cols, ld * 2, FK, FM, CU_TENSOR_MAP_SWIZZLE_128B);
+bool make_fit_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, rows, cols, ld * 2, FK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 template <int MODE>
@@ -460,7 +492,7 @@ struct FitScratch {
 };
 
 FitScratch carve_fit_scratch(unsigned char *base, int64_t M, int64_t d_out, int64_t d_in) {
-    const int64_t tiles_tok = (M + FN - 1) / FN, tiles_o = (d_out + FM - 1) / FM;
+    const int64_t tiles_tok = (M + fit_tokens(FIT_ROW_FWD) - 1) / fit_tokens(FIT_ROW_FWD), tiles_o = (d_out + FM - 1) / FM;  // the narrowest token tile
     const int64_t maxdim = d_out > d_in ? d_out : d_in;
     FitScratch s;
     size_t off = 0;
@@ -505,11 +537,12 @@ pd_status launch_fit_loss_grad(const __half *x, const __half *y, int64_t M, cons
                                const uint32_t *mask_t, const float *v, int axis, int64_t d_out, int64_t d_in, float *loss,
                                float *grad, unsigned char *scratch, uint32_t *status, cudaStream_t stream) {
     const FitScratch sc = carve_fit_scratch(scratch, M, d_out, d_in);
-    const int tiles_tok = static_cast<int>((M + FN - 1) / FN);
+    const int bn = fit_tokens(axis == PD_AXIS_COL ? FIT_COL_FWD : FIT_ROW_FWD);
+    const int tiles_tok = static_cast<int>((M + bn - 1) / bn);
     const int64_t ld_r = static_cast<int64_t>(round_up(static_cast<size_t>(d_out), 8));
     const double inv_n = 1.0 / (static_cast<double>(M) * static_cast<double>(d_out));
     CUtensorMap mw, mx;
-    if (!make_fit_map(&mw, w_b, d_out, d_in, d_in) || !make_fit_map(&mx, x, M, d_in, d_in)) return PD_ERR_CUDA;
+    if (!make_fit_map(&mw, w_b, d_out, d_in, d_in, FM) || !make_fit_map(&mx, x, M, d_in, d_in, bn)) return PD_ERR_CUDA;
     FitArgs a = {};
     a.bits = mask;
     a.words = static_cast<int>(d_in / 32);
@@ -546,7 +579,7 @@ pd_status launch_fit_loss_grad(const __half *x, const __half *y, int64_t M, cons
     int g_blocks = 0;
     if (grad) {
         CUtensorMap mr;
-        if (!make_fit_map(&mr, sc.resid, M, d_out, ld_r)) return PD_ERR_CUDA;
+        if (!make_fit_map(&mr, sc.resid, M, d_out, ld_r, fit_tokens(FIT_COL_BWD))) return PD_ERR_CUDA;
         FitArgs b = a;
         b.bits = mask_t;
         b.words = static_cast<int>((d_out + 31) / 32);
