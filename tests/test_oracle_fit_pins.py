@@ -189,7 +189,7 @@ def check_selection_keeps_the_lower_validation_loss():
     assert np.array_equal(v, vr if axis == ROW else vc)
     for a, vec, e in ((ROW, vr, e_row), (COL, vc, e_col)):
         again, _ = orc.loss_grad(x[32:], y[32:], w_b, mask, vec, a, want_grad=False)
-        assert again == e
+        assert abs(again - e) <= 1e-13 * e  # the OpenMP reduction adds the threads' partial sums in any order
 
 
 CHECKS = [v for k, v in sorted(globals().items()) if k.startswith("check_")]
