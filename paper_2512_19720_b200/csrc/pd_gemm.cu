@@ -838,11 +838,14 @@ splitk_reduce_kernel(const float *partial, int splits, int M, int d_out, __half 
     const float *src = partial + static_cast<size_t>(tok) * d_out + o;
     unsigned short *dst = reinterpret_cast<unsigned short *>(y) + static_cast<size_t>(tok) * ldy + o;
     if (vec_ok) {
-        float4 acc = *reinterpret_cast<const float4 *>(src);
-        for (int sp = 1; sp < splits; ++sp) {
-            const float4 t = *reinterpret_cast<const float4 *>(src + sp * plane);
-            acc.x += t.x, acc.y += t.y, acc.z += t.z, acc.w += t.w;
-        }
+        float4 part[8];  // all loads first (splits <= 8), then the sum in split order
+#pragma unroll
+        for (int sp = 0; sp < 8; ++sp)
+            part[sp] = sp < splits ? __ldcs(reinterpret_cast<const float4 *>(src + sp * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 acc = part[0];
+#pragma unroll
+        for (int sp = 1; sp < 8; ++sp)
+            if (sp < splits) acc.x += part[sp].x, acc.y += part[sp].y, acc.z += part[sp].z, acc.w += part[sp].w;
         uint2 out;
         out.x = Elem<BF16>::from_float(acc.x) | (static_cast<uint32_t>(Elem<BF16>::from_float(acc.y)) << 16);
         out.y = Elem<BF16>::from_float(acc.z) | (static_cast<uint32_t>(Elem<BF16>::from_float(acc.w)) << 16);
