@@ -279,7 +279,8 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                             const float yv = __half2float(ycol[(c0 + j) * FM]);
                             const float r = __uint_as_float(z[j]) - yv;
                             l_acc = fmaf(r, r, l_acc);
-                            a.resid[static_cast<size_t>(tok) * a.ld_r + row] = __float2half_rn(r);
+                            // the residual takes y's place in the shared-memory tile (this thread alone touches the entry)
+                            const_cast<__half *>(ycol)[(c0 + j) * FM] = __float2half_rn(r);
                         }
                     }
                 } else {
@@ -297,6 +298,16 @@ fit_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty);
+            if (MODE == FIT_COL_FWD) {  // the residual tile leaves with 16-byte stores, 256 contiguous bytes per token
+                asm volatile("bar.sync 2, %0;" ::"n"(kFitEpiWarps * 32) : "memory");
+                for (int idx = et; idx < count * 16; idx += kFitEpiWarps * 32) {
+                    const int tok = idx >> 4, ch = idx & 15;
+                    const int r8 = tm * FM + ch * 8;
+                    if (r8 < a.rows)
+                        *reinterpret_cast<uint4 *>(a.resid + static_cast<size_t>(tok0 + tok) * a.ld_r + r8) =
+                            *reinterpret_cast<const uint4 *>(ybuf + tok * (FM * 2) + ch * 16);
+                }
+            }
             if (MODE != FIT_COL_FWD && row_ok) a.part_g[static_cast<size_t>(tn) * a.rows + row] = g_acc;
             if (!FWD) asm volatile("bar.sync 2, %0;" ::"n"(kFitEpiWarps * 32) : "memory");  // the tile in shared memory is free again
             if (FWD) {  // squared error of the tile: lanes in a fixed tree, then the four warps in order
