@@ -13,9 +13,8 @@
 //                 error and the row gradient without writing R anywhere
 //   FIT_COL_FWD : one accumulator; the epilogue writes R as binary16 for the second pass
 //   FIT_COL_BWD : T^T = B^T R^T from the transposed mask (rows = input columns); the epilogue multiplies by X
-// A k step's cost is set by its TMA loads (128 row segments of W_b + one per token, ~3 clocks each) more than by its
-// MMAs, so the tiles are as wide in tokens as tensor memory allows in the row mode: 2 x 192 accumulator columns + the
-// sign ring (4 x 32).  The tile of Y (of X in the
+// About half of a k step's time does not depend on the number of tokens, so the tiles are as wide in tokens as tensor
+// memory allows in the row mode: 2 x 192 accumulator columns + the sign ring (4 x 32).  The tile of Y (of X in the
 // backward mode) that the epilogue needs is fetched into shared memory with cp.async while the tile's MMAs run:
 // read element by element from global memory it cost 40 % of the kernel's time.
 // The W_b tile is an MMA operand straight from the shared memory TMA filled (A from a shared-memory descriptor);

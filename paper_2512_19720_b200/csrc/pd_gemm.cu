@@ -1038,9 +1038,9 @@ pd_status launch_gemm_pair_grouped(const __half *x_sorted, int64_t M, const __ha
 
 namespace {
 
-// Token tile and number of k splits of the pair kernel.  A pair of k steps costs at least about 1250 clocks whatever
-// the tile's width (each CTA's TMA loads: 256 row segments of W_b and the x rows, ~3 clocks per segment) and the tensor
-// cores 4 clocks per token; a tile costs about 3000 clocks to start and drain.  With few tokens the tiles are too few for the 74 CTA pairs: the k steps are then
+// Token tile and number of k splits of the pair kernel.  Measured: a pair of k steps costs at least about 1250 clocks
+// whatever the tile's width, and 4 clocks per token plus 400 when that is more; a tile costs about 3000 clocks to
+// start and drain.  With few tokens the tiles are too few for the 74 CTA pairs: the k steps are then
 // dealt to several tiles whose fp32 partial sums a second kernel adds (about 5000 clocks plus its traffic).  Picks
 // the cheapest estimate; ties go to fewer splits, then to the narrower tile (more CTAs stream the weights).
 void pair_plan(int64_t M, int64_t d_out, int64_t d_in, int sms, int *token_tile, int *splits) {
