@@ -6,6 +6,7 @@ A step is one pass of the whole path, all through the C ABI, inputs resident in 
   Llama-7B-shaped decoder block (q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008)
     pack           pd_pack_delta on the 7 linears (mask + both scale vectors)
     decode_m*      pd_linear, M in {1, 4, 16} x {row, col} x 7 linears             <- headline metric
+    decode_par_m*  the same calls dealt to four streams (the linears of a sweep are independent: their kernels may overlap)
     prefill_m*     pd_linear, M in {256, 2048, 8192} x {row, col} x 7 linears
     multi_*        pd_linear_multivariant, 16 variants over one base: 64 decode rows; 64 + 4 x 512 rows with an id
                    per row; the same with one id per 512-row sequence; both batch sizes with mixed axes
@@ -362,6 +363,27 @@ def run_ours(args):
                 api.pd_linear(x_all[L["d_in"]][:m], L["w_b"], L["mask"], L["v"][axis], axis, y=y_all[L["d_out"]][:m],
                               weights_resident=resident)
 
+    PAR = 4  # parallel branches of the decode_par_* sections
+    par_streams = [torch.cuda.Stream(device=dev) for _ in range(PAR)]
+    par_y = [{d_out: torch.empty((16, d_out), dtype=torch.float16, device=dev) for d_out in (4096, 11008)} for _ in range(PAR)]
+
+    def run_linear_par(m):
+        # the same 14 calls as decode_m*, dealt to PAR streams: the linears of a sweep do not depend on one another (in a
+        # decoder block q, k, v share an input, and so do gate and up), so their kernels may overlap on the GPU
+        cur = torch.cuda.current_stream()
+        for ps in par_streams:
+            ps.wait_stream(cur)
+        i = 0
+        for axis in (ROW, COL):
+            for L in layers:
+                b = i % PAR
+                i += 1
+                with torch.cuda.stream(par_streams[b]):
+                    api.pd_linear(x_all[L["d_in"]][:m], L["w_b"], L["mask"], L["v"][axis], axis, y=par_y[b][L["d_out"]][:m],
+                                  weights_resident=True)
+        for ps in par_streams:
+            cur.wait_stream(ps)
+
     def run_multi(m, id_t, key, axes):
         for L in layers:
             api.pd_linear_multivariant(x_all[L["d_in"]][:m], id_t, L["w_b"], L["masks"], L[key], axes, y=y_all[L["d_out"]][:m])
@@ -429,6 +451,9 @@ def run_ours(args):
         add(f"decode_m{m}", lambda m=m: run_linear(m, True),
             sum(linear_bytes(m, L["d_out"], L["d_in"], ax) for ax in (ROW, COL) for L in layers), "GB/s", 14,
             "gemv_stream_kernel")
+    for m in DECODE_M:
+        add(f"decode_par_m{m}", lambda m=m: run_linear_par(m), S[f"decode_m{m}"]["work"], "GB/s", 14,
+            "gemv_stream_kernel, four streams")
     for m in PREFILL_M:
         add(f"prefill_m{m}", lambda m=m: run_linear(m, False), 2 * flops(m), "TFLOP/s", 14, "gemm_pair_kernel (tcgen05, CTA pairs)",
             bound="tensor" if m > 256 else "max(hbm, tensor)")
@@ -566,7 +591,53 @@ def run_ours(args):
         e2e_step()
     e1.record()
     barrier()
+    e2e_eager_ms = e0.elapsed_time(e1) / args.steps  # one host call per linear: the host's ~35 us per call is what this measures
+    # the same calls captured once into a CUDA graph (copy nodes from and to pinned host memory around every kernel) and
+    # replayed: what a serving loop does with a fixed decode step
+    # -- the calls of a step are independent, so the graph has E2E_BRANCHES parallel branches with their own staging and
+    # output buffers: one call's copies overlap the other branches' kernels (a copy over PCIe costs ~10 us whatever its size)
+    E2E_BRANCHES = 4
+    br_streams = [torch.cuda.Stream(device=dev) for _ in range(E2E_BRANCHES)]
+    br_dx = [{d_in: torch.empty((16, d_in), dtype=torch.float16, device=dev) for d_in in x_all} for _ in range(E2E_BRANCHES)]
+    br_y = [{d_out: torch.empty((16, d_out), dtype=torch.float16, device=dev) for d_out in y_all} for _ in range(E2E_BRANCHES)]
+    br_host_y = [{d_out: torch.empty((16, d_out), dtype=torch.float16).pin_memory() for d_out in y_all} for _ in range(E2E_BRANCHES)]
+
+    def e2e_step_branches():
+        cur = torch.cuda.current_stream()
+        for bs in br_streams:
+            bs.wait_stream(cur)
+        i = 0
+        for m in DECODE_M:
+            for axis in (ROW, COL):
+                for L in layers:
+                    b = i % E2E_BRANCHES
+                    i += 1
+                    with torch.cuda.stream(br_streams[b]):
+                        api.pd_linear_host(host_x[L["d_in"]][:m], br_dx[b][L["d_in"]], L["w_b"], L["mask"], L["v"][axis], axis,
+                                           br_y[b][L["d_out"]], br_host_y[b][L["d_out"]][:m], weights_resident=True)
+        for bs in br_streams:
+            cur.wait_stream(bs)
+
+    with torch.cuda.stream(side):
+        e2e_step_branches()  # eager once
+    torch.cuda.synchronize()
+    e2e_graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(e2e_graph, stream=side):
+            e2e_step_branches()
+    for _ in range(3):
+        e2e_graph.replay()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_graph.replay()
+    e1.record()
+    barrier()
     e2e_ms = e0.elapsed_time(e1) / args.steps
+    # the last replay's outputs reached the host buffers and equal the one-by-one run's (same inputs, same kernels)
+    last = len(DECODE_M) * 2 * len(layers) - 1
+    assert torch.equal(br_host_y[last % E2E_BRANCHES][layers[-1]["d_out"]][:DECODE_M[-1]], host_y[layers[-1]["d_out"]][:DECODE_M[-1]])
 
     # ---- cold start (pd_load_merged): the delta artifacts of N_LOAD_LAYERS blocks in pinned host memory are copied
     # module by module while the previous module is merged into the resident base; beside it, the same bytes of
@@ -679,7 +750,10 @@ def run_ours(args):
             "rooflines": all_roofs,
             "e2e": {"value": round(dec_work * world / (e2e_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
-                    "what": "decode sections through pd_linear_host: x from pinned host memory, y back to pinned host memory, every call"},
+                    "eager_value": round(dec_work * world / (e2e_eager_ms * 1e-3) / 1e9, 1), "eager_ms_per_step": round(e2e_eager_ms, 4),
+                    "what": "decode sections through pd_linear_host: x from pinned host memory, y back to pinned host memory, every "
+                            "call; `value` replays the step's calls from a CUDA graph of four parallel branches (copies included; the calls "
+                            "are independent), `eager_value` issues them one by one on one stream"},
             "cold_start": {"what": f"{N_LOAD_LAYERS} 7B blocks ({len(load_mods)} modules): pd_load_merged from pinned host artifacts "
                                    "(H2D of module i+1 overlaps the merge of module i) against an H2D copy of the dense fp16 weights",
                            "delta_ms": round(load_ms["delta_on_resident_base"], 3), "delta_artifact_bytes": art_bytes,
