@@ -6,7 +6,8 @@ A step is one pass of the whole path, all through the C ABI, inputs resident in 
   Llama-7B-shaped decoder block (q/k/v/o 4096x4096, gate/up 11008x4096, down 4096x11008)
     pack           pd_pack_delta on the 7 linears (mask + both scale vectors)
     decode_m*      pd_linear, M in {1, 4, 16} x {row, col} x 7 linears             <- headline metric
-    decode_par_m*  the same calls dealt to four streams (the linears of a sweep are independent: their kernels may overlap)
+    *_par*         decode, pack, merge and prefill M = 256 with the sweep's calls dealt to four streams (the linears of a
+                   sweep are independent: their kernels may overlap)
     prefill_m*     pd_linear, M in {256, 2048, 8192} x {row, col} x 7 linears
     multi_*        pd_linear_multivariant, 16 variants over one base: 64 decode rows; 64 + 4 x 512 rows with an id
                    per row; the same with one id per 512-row sequence; both batch sizes with mixed axes
@@ -384,6 +385,38 @@ def run_ours(args):
         for ps in par_streams:
             cur.wait_stream(ps)
 
+    def on_branches(calls):
+        """Deals the calls (callables taking the branch index) to the PAR streams and joins them."""
+        cur = torch.cuda.current_stream()
+        for ps in par_streams:
+            ps.wait_stream(cur)
+        for i, call in enumerate(calls):
+            with torch.cuda.stream(par_streams[i % PAR]):
+                call(i % PAR)
+        for ps in par_streams:
+            cur.wait_stream(ps)
+
+    # pack and the split-K prefill use scratch memory: one workspace per branch (the pack's starts zeroed and is left zeroed)
+    par_pack_ws = [torch.zeros(max(api.workspace_bytes(api.OP_PACK, 0, 0, L["d_out"], L["d_in"]) for L in layers), dtype=torch.uint8,
+                               device=dev) for _ in range(PAR)]
+    par_lin_ws = [torch.zeros(max(api.workspace_bytes(api.OP_LINEAR, 256, 0, L["d_out"], L["d_in"]) for L in layers), dtype=torch.uint8,
+                              device=dev) for _ in range(PAR)]
+    par_y256 = [{d_out: torch.empty((256, d_out), dtype=torch.float16, device=dev) for d_out in (4096, 11008)} for _ in range(PAR)]
+
+    def run_pack_par():
+        on_branches([lambda b, L=L: api.pd_pack_delta(L["w_f"], L["w_b"], mask=L["mask"], v_row=L["v"][0], v_col=L["v"][1],
+                                                      workspace=par_pack_ws[b]) for L in layers])
+
+    def run_merge_par():
+        # both axes write the layer's one w_hat buffer: one axis per layer here, so that no two branches share an output
+        on_branches([lambda b, L=L, axis=axis: api.pd_merge(L["w_b"], L["mask"], L["v"][axis], axis, w_hat=L["w_hat"])
+                     for axis, L in zip([ROW, COL] * len(layers), layers)])
+
+    def run_prefill256_par():
+        on_branches([lambda b, L=L, axis=axis: api.pd_linear(x_all[L["d_in"]][:256], L["w_b"], L["mask"], L["v"][axis], axis,
+                                                             y=par_y256[b][L["d_out"]], workspace=par_lin_ws[b])
+                     for axis in (ROW, COL) for L in layers])
+
     def run_multi(m, id_t, key, axes):
         for L in layers:
             api.pd_linear_multivariant(x_all[L["d_in"]][:m], id_t, L["w_b"], L["masks"], L[key], axes, y=y_all[L["d_out"]][:m])
@@ -454,6 +487,11 @@ def run_ours(args):
     for m in DECODE_M:
         add(f"decode_par_m{m}", lambda m=m: run_linear_par(m), S[f"decode_m{m}"]["work"], "GB/s", 14,
             "gemv_stream_kernel, four streams")
+    add("pack_par", run_pack_par, S["pack"]["work"], "GB/s", 7, "pack_kernel, four streams")
+    add("merge_par", run_merge_par, sum(merge_bytes(L["d_out"], L["d_in"], ax) for ax, L in zip([ROW, COL] * len(layers), layers)), "GB/s", 7,
+        "merge_kernel, four streams")
+    add("prefill_par_m256", run_prefill256_par, 2 * flops(256), "TFLOP/s", 14, "gemm_pair_kernel (split-K), four streams",
+        bound="max(hbm, tensor)")
     for m in PREFILL_M:
         add(f"prefill_m{m}", lambda m=m: run_linear(m, False), 2 * flops(m), "TFLOP/s", 14, "gemm_pair_kernel (tcgen05, CTA pairs)",
             bound="tensor" if m > 256 else "max(hbm, tensor)")
