@@ -13,7 +13,7 @@
  * the merged form):
  *
  *   dW      = W_f - W_b                              (exact in fp64 for fp16 inputs)
- *   B       = sign(dW) in {-1,+1}; this build reads sign(0) as +1
+ *   B       = sign(dW) in {-1,+1}; sign(0) is read as +1 (the Method section leaves it open)
  *   mask    : B packed 1 bit per entry along the input axis, 32 entries per uint32,
  *             bit k of word w of row o  <->  column 32*w + k, bit 1 <-> +1
  *   v_row[o]= mean_i |dW[o,i]|   (length d_out)      v_col[i] = mean_o |dW[o,i]| (length d_in)
