@@ -60,7 +60,7 @@ ROW, COL = 0, 1
 # elements streamed).  Pack and multi-variant decode: read + write.  Decode GEMV and merge: the read ratio -- the GEMV
 # writes 8 KB, what ncu counts as its writes is earlier data leaving the L2, and half of merge's writes are still dirty
 # in L2 when the kernel ends.  None = the kernel has changed since its counters were taken.
-NCU_DRAM_RATIO = {"decode": 1.004, "pack": 0.996, "merge": 1.0, "multi_decode": 0.987}
+NCU_DRAM_RATIO = {"decode": 1.004, "pack": 1.0, "merge": 1.0, "multi_decode": 0.987}
 METRIC = "fused delta-linear decode HBM GB/s (7B block sweep, M in {1,4,16}, row+col axes)"
 
 
